@@ -1,0 +1,482 @@
+"""Pins for the CPU oracle: each test checks an oracle function against something other than
+itself - a value the paper prints, a closed form, a textbook/library routine, an invariant, or a
+brute-force search on tiny inputs."""
+import math
+import os
+
+import numpy as np
+import pytest
+import scipy.special
+import torch
+
+import oracle
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+rng = np.random.default_rng(20250607)
+
+
+def to_bf16_bits(a):
+    t = torch.tensor(np.asarray(a, dtype=np.float32)).to(torch.bfloat16)
+    return t.view(torch.int16).numpy().view(np.uint16)
+
+
+# ------------------------------------------------------------------------------ number format
+def test_bf16_decode_known_patterns():
+    bits = np.array([0x3F80, 0xC000, 0x0000, 0x3DCD, 0x7F7F, 0x8000], dtype=np.uint16)
+    got = oracle.bf16_bits_to_f64(bits)
+    want = [1.0, -2.0, 0.0, 0.10009765625, 3.3895313892515355e38, -0.0]
+    assert got.tolist() == want
+    assert math.copysign(1.0, got[-1]) == -1.0
+
+
+def test_bf16_decode_matches_torch():
+    bits = rng.integers(0, 1 << 16, size=4096, dtype=np.uint16)
+    bits = bits[(bits & 0x7F80) != 0x7F80]          # finite values only
+    t = torch.from_numpy(bits.view(np.int16).copy()).view(torch.bfloat16).to(torch.float64)
+    assert np.array_equal(oracle.bf16_bits_to_f64(bits), t.numpy())
+
+
+# ------------------------------------------------------------------------------ route
+def brute_force_topk(logits_row, K):
+    """Repeatedly extract the maximum; among equal values the lower index wins."""
+    left = list(range(len(logits_row)))
+    out = []
+    for _ in range(K):
+        best = left[0]
+        for e in left[1:]:
+            if logits_row[e] > logits_row[best]:
+                best = e
+        out.append(best)
+        left.remove(best)
+    return out
+
+
+def test_route_logits_one_hot_closed_form():
+    # X rows are unit vectors: logit[t, e] must be Wr[e, d_t] + b[e] (catches a transposed operand).
+    T, D, E = 5, 7, 3
+    d_of_t = [6, 0, 3, 3, 1]
+    X = np.zeros((T, D))
+    for t, d in enumerate(d_of_t):
+        X[t, d] = 1.0
+    Wr = oracle.bf16_bits_to_f64(to_bf16_bits(rng.normal(size=(E, D))))
+    b = rng.normal(size=E).astype(np.float32)
+    got = oracle.route_logits(to_bf16_bits(X), to_bf16_bits(Wr), b)
+    for t, d in enumerate(d_of_t):
+        for e in range(E):
+            assert got[t, e] == Wr[e, d] + float(b[e])
+
+
+@pytest.mark.parametrize("E,K,mode", [(8, 2, 0), (8, 8, 0), (16, 1, 0), (32, 6, 1), (5, 3, 1)])
+def test_route_selection_brute_force(E, K, mode):
+    T, D = 64, 24
+    x = to_bf16_bits(rng.normal(size=(T, D)))
+    wr = to_bf16_bits(rng.normal(size=(E, D)) / math.sqrt(D))
+    b = rng.normal(size=E).astype(np.float32)
+    idx, w, logits = oracle.route(x, wr, b, K, mode)
+    assert idx.shape == (T, K) and w.shape == (T, K) and idx.dtype == np.int32
+    for t in range(T):
+        assert idx[t].tolist() == brute_force_topk(logits[t], K)
+    assert np.allclose(w.sum(axis=1), 1.0, atol=1e-12)
+    assert (w > 0).all()
+
+
+def test_route_full_softmax_when_k_equals_e():
+    T, D, E = 16, 12, 6
+    x = to_bf16_bits(rng.normal(size=(T, D)))
+    wr = to_bf16_bits(rng.normal(size=(E, D)))
+    idx, w, logits = oracle.route(x, wr, None, E, 0)
+    full = scipy.special.softmax(logits, axis=1)
+    assert np.allclose(w, np.take_along_axis(full, idx.astype(np.int64), axis=1), rtol=1e-12)
+
+
+def test_route_softmax_is_full_softmax_renormalised():
+    T, D, E, K = 16, 12, 9, 3
+    x = to_bf16_bits(rng.normal(size=(T, D)))
+    wr = to_bf16_bits(rng.normal(size=(E, D)))
+    idx, w, logits = oracle.route(x, wr, None, K, 0)
+    full = scipy.special.softmax(logits, axis=1)
+    sel = np.take_along_axis(full, idx.astype(np.int64), axis=1)
+    assert np.allclose(w, sel / sel.sum(axis=1, keepdims=True), rtol=1e-12)
+
+
+def test_route_sigmoid_mode_ratios():
+    T, D, E, K = 16, 12, 9, 4
+    x = to_bf16_bits(rng.normal(size=(T, D)))
+    wr = to_bf16_bits(rng.normal(size=(E, D)))
+    b = rng.normal(size=E).astype(np.float32)
+    idx, w, logits = oracle.route(x, wr, b, K, 1)
+    s = scipy.special.expit(np.take_along_axis(logits, idx.astype(np.int64), axis=1))
+    assert np.allclose(w * s.sum(axis=1, keepdims=True), s, rtol=1e-12)
+    # descending logits => descending weights in both modes
+    assert (np.diff(w, axis=1) <= 0).all()
+
+
+def test_route_k1_weight_is_one():
+    x = to_bf16_bits(rng.normal(size=(8, 4)))
+    wr = to_bf16_bits(rng.normal(size=(3, 4)))
+    for mode in (0, 1):
+        idx, w, logits = oracle.route(x, wr, None, 1, mode)
+        assert np.array_equal(w, np.ones((8, 1)))
+        assert np.array_equal(idx[:, 0], logits.argmax(axis=1))
+
+
+def test_route_exact_ties_go_to_lower_index():
+    T, D, E = 32, 16, 6
+    wr = rng.normal(size=(E, D))
+    wr[4] = wr[1]                       # experts 1 and 4 always tie exactly
+    wr[5] = wr[0]                       # experts 0 and 5 too
+    x = to_bf16_bits(rng.normal(size=(T, D)))
+    idx, w, logits = oracle.route(x, to_bf16_bits(wr), None, 3, 0)
+    for t in range(T):
+        sel = idx[t].tolist()
+        if 4 in sel:
+            assert 1 in sel and sel.index(1) < sel.index(4)
+        if 5 in sel:
+            assert 0 in sel and sel.index(0) < sel.index(5)
+    assert any(4 in idx[t] or 5 in idx[t] for t in range(T))
+
+
+def test_route_expert_permutation_equivariance():
+    T, D, E, K = 32, 16, 8, 3
+    x = to_bf16_bits(rng.normal(size=(T, D)))
+    wr = to_bf16_bits(rng.normal(size=(E, D)))
+    b = rng.normal(size=E).astype(np.float32)
+    perm = rng.permutation(E)
+    idx, w, _ = oracle.route(x, wr, b, K, 0)
+    idx2, w2, _ = oracle.route(x, wr[perm], b[perm], K, 0)
+    assert np.array_equal(perm[idx2], idx)
+    assert np.allclose(w2, w, rtol=1e-12)
+
+
+# ------------------------------------------------------------------------------ histogram / stats
+def test_histogram_against_bincount_and_sum():
+    T, K, E = 300, 3, 11
+    idx = rng.integers(0, E, size=(T, K)).astype(np.int32)
+    h = oracle.histogram(idx, E)
+    assert h.sum() == T * K
+    assert np.array_equal(h, np.bincount(idx.reshape(-1), minlength=E))
+    with pytest.raises(ValueError):
+        oracle.histogram(np.array([[0, E]]), E)
+    with pytest.raises(ValueError):
+        oracle.histogram(np.array([[-1, 0]]), E)
+    assert oracle.histogram(np.zeros((0, 2), dtype=np.int32), 4).tolist() == [0, 0, 0, 0]
+
+
+def test_skewness_paper_example():
+    rows = [l.split() for l in open(os.path.join(HERE, "golden", "skewness_example.txt"))
+            if l.strip() and not l.startswith("#")]
+    share, n_exp, want = float(rows[0][0]), int(rows[0][1]), float(rows[0][2])
+    total = 1200
+    top = int(round(share * total))
+    rest = (total - top) // (n_exp - 1)
+    hist = [top] + [rest] * (n_exp - 1)
+    assert sum(hist) == total
+    assert oracle.skewness(hist) == want
+    assert oracle.skewness([7, 7, 7, 7, 7]) == 1.0
+
+
+def test_p_hat_and_error_rate():
+    h = np.array([6, 3, 1, 0])
+    p = oracle.p_hat(h)
+    assert p.tolist() == [0.6, 0.3, 0.1, 0.0] and abs(p.sum() - 1) < 1e-15
+    assert oracle.error_rate(p, p) == 0.0
+    # hand-worked: E = 4, estimate (1/2, 1/2, 0, 0) against the uniform truth: every expert is off
+    # by 1/4 = one unit of 1/E, so the average is exactly 1.
+    assert oracle.error_rate([0.5, 0.5, 0.0, 0.0], [0.25] * 4) == 1.0
+    # one expert off by 0.1 up, another 0.1 down, E = 5: (0.1 + 0.1) / 5 / (1/5) = 0.2
+    assert abs(oracle.error_rate([0.3, 0.1, 0.2, 0.2, 0.2], [0.2] * 5) - 0.2) < 1e-15
+
+
+# ------------------------------------------------------------------------------ plan
+def compositions(total, parts):
+    """All ways to write `total` as an ordered sum of `parts` non-negative integers."""
+    if parts == 1:
+        yield (total,)
+        return
+    for first in range(total + 1):
+        for rest in compositions(total - first, parts - 1):
+            yield (first,) + rest
+
+
+def check_plan_tables(r, slot_off, slot_expert, S):
+    E = len(r)
+    assert (r >= 1).all() and slot_off[0] == 0
+    assert np.array_equal(np.diff(slot_off), r)
+    for e in range(E):
+        assert (slot_expert[slot_off[e]:slot_off[e + 1]] == e).all()
+    assert (slot_expert[slot_off[E]:] == -1).all()
+    assert slot_off[E] <= S
+
+
+def test_plan_minmax_optimal_brute_force():
+    from fractions import Fraction
+    for E in (1, 2, 3, 4, 5):
+        for extra in range(0, 6):
+            for _ in range(6):
+                n = rng.integers(0, 40, size=E)
+                r, so, se, bound = oracle.plan(n, E + extra)
+                check_plan_tables(r, so, se, E + extra)
+                assert r.sum() == E + extra
+                got = max(Fraction(int(n[e]), int(r[e])) for e in range(E))
+                best = min(max(Fraction(int(n[e]), 1 + c[e]) for e in range(E))
+                           for c in compositions(extra, E))
+                assert got == best
+                assert bound == max(-(-int(n[e]) // int(r[e])) for e in range(E))
+
+
+def test_plan_proportional_closed_form():
+    # predicted counts proportional to an integer composition of S: the balanced plan is that
+    # composition (Algorithm 1 stops when all devices carry the same load).
+    for c in (1, 7, 1000):
+        r, so, se, bound = oracle.plan(np.array([9, 1, 1, 1]) * c, 12)
+        assert r.tolist() == [9, 1, 1, 1] and bound == c
+    m = np.array([3, 1, 4, 1, 5, 2])
+    r, _, _, bound = oracle.plan(m * 13, int(m.sum()))
+    assert r.tolist() == m.tolist() and bound == 13
+
+
+def test_plan_hand_worked_ties_and_order():
+    assert oracle.plan([4, 2], 3)[0].tolist() == [2, 1]
+    assert oracle.plan([2, 2], 3)[0].tolist() == [2, 1]          # equal ratio, equal r: lower index
+    assert oracle.plan([4, 2], 4)[0].tolist() == [2, 2]          # 4/2 = 2/1: smaller r wins
+    assert oracle.plan([0, 0, 0], 8)[0].tolist() == [3, 3, 2]    # all-zero prediction: round robin
+    r, so, se, bound = oracle.plan([5, 0, 1], 5)
+    assert r.tolist() == [3, 1, 1] and so.tolist() == [0, 3, 4, 5]
+    assert se.tolist() == [0, 0, 0, 1, 2] and bound == 2
+    assert oracle.plan([3, 3, 3], 3)[0].tolist() == [1, 1, 1]    # S = E: no duplication
+
+
+def test_plan_copy_cap():
+    r, so, se, bound = oracle.plan([100, 1, 1], 8, c_max=3)
+    assert r.tolist() == [3, 3, 2]
+    r, so, se, bound = oracle.plan([100, 1], 8, c_max=2)
+    assert r.tolist() == [2, 2] and se.tolist() == [0, 0, 1, 1, -1, -1, -1, -1]
+    assert bound == 50
+    check_plan_tables(r, so, se, 8)
+
+
+def test_plan_bound_sandwich_and_monotone():
+    for _ in range(50):
+        E = int(rng.integers(2, 40))
+        n = rng.integers(0, 5000, size=E)
+        N = int(n.sum())
+        prev = None
+        for S in range(E, E + 12):
+            bound = oracle.plan(n, S)[3]
+            assert bound >= -(-N // S)
+            assert bound <= int(n.max())
+            if S > E:
+                assert bound <= max(1, -(-N // (S - E))) or N == 0
+            if prev is not None:
+                assert bound <= prev
+            prev = bound
+
+
+# ------------------------------------------------------------------------------ dispatch
+def closed_form_replica(i, n, r):
+    return ((i + 1) * r - 1) // n
+
+
+def random_routing(T, K, E, skew=1.0):
+    p = 1.0 / np.arange(1, E + 1) ** skew
+    p /= p.sum()
+    idx = np.stack([rng.choice(E, size=K, replace=False, p=p) for _ in range(T)]).astype(np.int32)
+    return idx
+
+
+@pytest.mark.parametrize("T,K,E,S,A", [(50, 2, 4, 4, 1), (50, 2, 4, 9, 1), (97, 3, 7, 12, 8),
+                                       (64, 1, 5, 5, 128), (33, 4, 4, 16, 4), (0, 2, 3, 5, 2)])
+def test_dispatch_invariants(T, K, E, S, A):
+    idx = random_routing(T, K, E, 1.3) if T else np.zeros((0, K), dtype=np.int32)
+    hist = oracle.histogram(idx, E)
+    r, so, se, bound = oracle.plan(hist, S)            # perfect prediction
+    D = 6
+    x = rng.integers(0, 1 << 16, size=(T, D), dtype=np.uint16)
+    sro, row_pair, pair_row, xp = oracle.dispatch(x, idx, hist, r, so, S, A)
+    R = T * K
+    Rcap = R + S * (A - 1)
+    assert row_pair.shape == (Rcap,) and pair_row.shape == (T, K) and xp.shape == (Rcap, D)
+    flat_rows = pair_row.reshape(-1)
+    # bijection between pairs and occupied rows
+    assert len(set(flat_rows.tolist())) == R
+    assert np.array_equal(row_pair[flat_rows], np.arange(R))
+    assert (row_pair >= 0).sum() == R
+    # slot structure
+    assert sro[0] == 0 and (np.diff(sro) >= 0).all() and (sro[:-1] % A == 0).all()
+    loads = []
+    for s in range(S):
+        rows = np.arange(sro[s], sro[s + 1])
+        occ = rows[row_pair[rows] >= 0]
+        loads.append(len(occ))
+        if len(occ):
+            assert occ[0] == sro[s] and np.array_equal(occ, np.arange(sro[s], sro[s] + len(occ)))
+            pairs = row_pair[occ]
+            assert (np.diff(pairs) > 0).all()                       # stable inside a slot
+            assert (idx.reshape(-1)[pairs] == se[s]).all()          # right expert
+    for e in range(E):
+        mine = loads[so[e]:so[e + 1]]
+        assert sum(mine) == hist[e]
+        assert all(l in (hist[e] // r[e], -(-hist[e] // r[e])) for l in mine)
+    assert max(loads + [0]) == (bound if R else 0)                  # perfect prediction: tight
+    # replica of a pair follows the closed form floor(((i+1) r - 1) / n)
+    seen = [0] * E
+    for p in range(R):
+        e = int(idx.reshape(-1)[p])
+        rho = closed_form_replica(seen[e], int(hist[e]), int(r[e]))
+        seen[e] += 1
+        assert sro[so[e] + rho] <= flat_rows[p] < sro[so[e] + rho + 1]
+    # rows are bit copies
+    for p in range(R):
+        assert np.array_equal(xp[flat_rows[p]], x[p // K])
+
+
+def test_dispatch_is_stable_sort_when_unreplicated():
+    T, K, E = 200, 2, 8
+    idx = random_routing(T, K, E, 1.0)
+    hist = oracle.histogram(idx, E)
+    r, so, se, _ = oracle.plan(hist, E)
+    sro, row_pair, pair_row, _ = oracle.dispatch(None, idx, hist, r, so, E, 1)
+    order = np.argsort(idx.reshape(-1), kind="stable")
+    assert np.array_equal(row_pair, order)
+    assert np.array_equal(sro, np.concatenate([[0], np.cumsum(hist)]))
+
+
+def test_dispatch_load_bound_under_misprediction():
+    # slot load <= ceil((1 + delta_e) * predicted_e / r_e): the slot-level form of the paper's
+    # "typical" (1 + eps) * average model of Section 3.3.
+    T, K, E, S = 400, 2, 8, 14
+    idx = random_routing(T, K, E, 1.2)
+    hist = oracle.histogram(idx, E)
+    pred = np.maximum(1, np.round(hist * (1 + 0.2 * rng.normal(size=E)))).astype(np.int64)
+    r, so, se, bound = oracle.plan(pred, S)
+    sro, row_pair, _, _ = oracle.dispatch(None, idx, hist, r, so, S, 1)
+    loads = np.diff(sro)
+    for e in range(E):
+        delta = max(0.0, hist[e] / pred[e] - 1.0)
+        for s in range(so[e], so[e + 1]):
+            assert loads[s] <= math.ceil((1 + delta) * pred[e] / r[e] + 1e-9)
+
+
+def test_dispatch_rejects_wrong_hist():
+    idx = random_routing(10, 2, 4)
+    hist = oracle.histogram(idx, 4)
+    hist[0] += 1
+    with pytest.raises(ValueError):
+        oracle.dispatch(None, idx, hist, [1] * 4, [0, 1, 2, 3, 4], 4, 1)
+
+
+# ------------------------------------------------------------------------------ expert_ffn / combine
+def tiny_layer(T=24, D=16, F=24, E=4, K=2):
+    x = to_bf16_bits(rng.normal(size=(T, D)))
+    wr = to_bf16_bits(rng.normal(size=(E, D)) / math.sqrt(D))
+    b = rng.normal(size=E).astype(np.float32)
+    w1 = to_bf16_bits(rng.normal(size=(E, F, D)) * 0.3)
+    w3 = to_bf16_bits(rng.normal(size=(E, F, D)) * 0.3)
+    w2 = to_bf16_bits(rng.normal(size=(E, D, F)) * 0.3)
+    return x, wr, b, w1, w3, w2
+
+
+def dense_then_mask(x, wr, b, w1, w3, w2, K, mode):
+    """Every expert on every token with torch's own SiLU, then the K-sparse gate matrix."""
+    X = torch.from_numpy(oracle.bf16_bits_to_f64(x))
+    E = wr.shape[0]
+    idx, w, _ = oracle.route(x, wr, b, K, mode)
+    gate = torch.zeros(X.shape[0], E, dtype=torch.float64)
+    for t in range(X.shape[0]):
+        for j in range(K):
+            gate[t, idx[t, j]] = w[t, j]
+    out = torch.zeros(X.shape[0], w2.shape[1], dtype=torch.float64)
+    for e in range(E):
+        W1 = torch.from_numpy(oracle.bf16_bits_to_f64(w1[e]))
+        W3 = torch.from_numpy(oracle.bf16_bits_to_f64(w3[e]))
+        W2 = torch.from_numpy(oracle.bf16_bits_to_f64(w2[e]))
+        y = (torch.nn.functional.silu(X @ W1.T) * (X @ W3.T)) @ W2.T
+        out += gate[:, e:e + 1] * y
+    return out.numpy()
+
+
+@pytest.mark.parametrize("S,A,mode,pred", [(4, 1, 0, "true"), (7, 1, 0, "zero"), (9, 4, 1, "true"),
+                                           (6, 128, 0, "skewed")])
+def test_layer_equals_dense_all_experts_then_mask(S, A, mode, pred):
+    x, wr, b, w1, w3, w2 = tiny_layer()
+    E, K = 4, 2
+    true_hist = oracle.histogram(oracle.route(x, wr, b, K, mode)[0], E)
+    pred_hist = {"true": true_hist, "zero": np.zeros(E, dtype=np.int64),
+                 "skewed": np.array([100, 0, 3, 1])}[pred]
+    res = oracle.moe_layer(x, wr, b, w1, w3, w2, pred_hist, K=K, S=S, gate_mode=mode, row_align=A)
+    want = dense_then_mask(x, wr, b, w1, w3, w2, K, mode)
+    assert np.allclose(res["out"], want, rtol=1e-10, atol=1e-12)
+    assert res["hist"].sum() == x.shape[0] * K
+
+
+def test_layer_output_independent_of_placement():
+    x, wr, b, w1, w3, w2 = tiny_layer()
+    base = oracle.moe_layer(x, wr, b, w1, w3, w2, [1, 1, 1, 1], K=2, S=4)["out"]
+    for S, A, c_max, pred in [(11, 1, 0, [50, 1, 1, 1]), (8, 16, 2, [0, 9, 0, 9]), (5, 3, 0, [1, 2, 3, 4])]:
+        out = oracle.moe_layer(x, wr, b, w1, w3, w2, pred, K=2, S=S, row_align=A, c_max=c_max)["out"]
+        assert np.allclose(out, base, rtol=1e-12, atol=1e-14)
+
+
+def test_ffn_single_expert_is_a_dense_mlp():
+    T, D, F = 10, 8, 12
+    xp = to_bf16_bits(rng.normal(size=(T, D)))
+    w1 = to_bf16_bits(rng.normal(size=(1, F, D)))
+    w3 = to_bf16_bits(rng.normal(size=(1, F, D)))
+    w2 = to_bf16_bits(rng.normal(size=(1, D, F)))
+    yp = oracle.expert_ffn(xp, [0, T], [0], w1, w3, w2)
+    X = torch.from_numpy(oracle.bf16_bits_to_f64(xp))
+    lin1 = torch.nn.Linear(D, F, bias=False, dtype=torch.float64)
+    lin3 = torch.nn.Linear(D, F, bias=False, dtype=torch.float64)
+    lin2 = torch.nn.Linear(F, D, bias=False, dtype=torch.float64)
+    with torch.no_grad():
+        lin1.weight.copy_(torch.from_numpy(oracle.bf16_bits_to_f64(w1[0])))
+        lin3.weight.copy_(torch.from_numpy(oracle.bf16_bits_to_f64(w3[0])))
+        lin2.weight.copy_(torch.from_numpy(oracle.bf16_bits_to_f64(w2[0])))
+        want = lin2(torch.nn.functional.silu(lin1(X)) * lin3(X)).numpy()
+    assert np.allclose(yp, want, rtol=1e-12, atol=1e-14)
+
+
+def test_ffn_zero_weights_and_row_subset():
+    T, D, F, E = 12, 8, 10, 3
+    xp = to_bf16_bits(rng.normal(size=(T, D)))
+    w1 = to_bf16_bits(rng.normal(size=(E, F, D)))
+    w3 = to_bf16_bits(rng.normal(size=(E, F, D)))
+    w2 = to_bf16_bits(rng.normal(size=(E, D, F)))
+    off, se = [0, 5, 5, 12], [2, 0, 1]
+    full = oracle.expert_ffn(xp, off, se, w1, w3, w2)
+    assert np.abs(full).max() > 0
+    assert not oracle.expert_ffn(xp, off, se, np.zeros_like(w1), w3, w2).any()   # silu(0) = 0
+    assert not oracle.expert_ffn(xp, off, se, w1, w3, np.zeros_like(w2)).any()
+    part = oracle.expert_ffn(xp, off, se, w1, w3, w2, rows=[1, 7, 11])
+    assert np.allclose(part[[1, 7, 11]], full[[1, 7, 11]], rtol=1e-12, atol=0)
+    assert not part[[0, 2, 3, 4, 5, 6, 8, 9, 10]].any()
+    # each slot uses its own expert: swapping the experts of two slots changes those rows only
+    swapped = oracle.expert_ffn(xp, off, [1, 0, 2], w1, w3, w2)
+    assert not np.allclose(swapped, full)
+
+
+def test_combine_identity_gather_and_linearity():
+    T, K, E, D = 40, 3, 6, 8
+    idx = random_routing(T, K, E)
+    hist = oracle.histogram(idx, E)
+    r, so, se, _ = oracle.plan(hist, 9)
+    x = to_bf16_bits(rng.normal(size=(T, D)))
+    sro, row_pair, pair_row, xp = oracle.dispatch(x, idx, hist, r, so, 9, 4)
+    w = rng.random(size=(T, K))
+    w /= w.sum(axis=1, keepdims=True)
+    # Yp := Xp with weights that sum to one gives back X
+    out = oracle.combine(xp, pair_row, w)
+    assert np.allclose(out, oracle.bf16_bits_to_f64(x), rtol=1e-12, atol=1e-15)
+    # K = 1: a pure gather
+    out1 = oracle.combine(xp, pair_row[:, :1], np.ones((T, 1)))
+    assert np.array_equal(out1, oracle.bf16_bits_to_f64(x))
+    # linear in the weights, and a hand-checkable case
+    yp = rng.normal(size=(xp.shape[0], D))
+    w2 = rng.random(size=(T, K))
+    assert np.allclose(oracle.combine(yp, pair_row, 2 * w + 3 * w2),
+                       2 * oracle.combine(yp, pair_row, w) + 3 * oracle.combine(yp, pair_row, w2))
+    small = oracle.combine(np.array([[1.0, 10.0], [2.0, 20.0], [4.0, 40.0]]),
+                           np.array([[2, 0]]), np.array([[0.25, 0.5]]))
+    assert small.tolist() == [[1.5, 15.0]]
+    sub = oracle.combine(yp, pair_row, w, tokens=[3, 17])
+    assert np.array_equal(sub[[3, 17]], oracle.combine(yp, pair_row, w)[[3, 17]])
