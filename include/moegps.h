@@ -1,0 +1,172 @@
+/*
+ * moegps.h - C ABI of the B200 (sm_100a) hot path of one Mixture-of-Experts inference layer with
+ * prediction-driven expert duplication.
+ *
+ * The layer is the one whose load balance the MoE-GPS paper studies: tokens are routed to their
+ * top-K experts (paper, Section 2), the per-expert token counts form the distribution that
+ * Distribution-Only Prediction forecasts (Section 3.2.1, Eq. 1), a duplication plan replicates
+ * popular experts (Section 3.1, Algorithm 1), tokens are shuffled to the replica that serves them
+ * (the routing all-to-all of Section 2), the experts' SwiGLU FFNs run (Sections 2 and 3.4), and the
+ * results are shuffled back to token order (last sentence of the communication paragraph of
+ * Section 2).  Here all of it runs on ONE device: the "GPUs" of Algorithm 1 become S logical slots,
+ * each holding one expert replica and owning a contiguous bucket of rows.
+ *
+ * Notation: T tokens, D model width, F expert hidden width, E experts, K experts per token,
+ * S slots (S >= E), R = T*K routed pairs with flat index p = t*K + j, A = row_align,
+ * Rcap = R + S*(A-1) rows in the permuted buffers.
+ *
+ * Conventions that hold for every call
+ *  - Every tensor pointer is a DEVICE pointer owned by the caller, 16-byte aligned, row-major with
+ *    the last dimension contiguous.  bf16 tensors are passed as `const void*` / `void*`.
+ *  - The library allocates no device memory after moegps_create, copies nothing to the host and
+ *    never synchronises, except in moegps_status.  `stream` is a cudaStream_t passed as void*
+ *    (NULL = the legacy default stream).  Calls are asynchronous and ordered by the stream.
+ *  - Outputs are fully overwritten unless stated; inputs are never modified.
+ *  - Return value: MOEGPS_OK (0) or a negative moegps_error code.  Arguments are validated on the
+ *    host before anything is launched; a failing call launches nothing.  Conditions only the device
+ *    can see (an expert index out of range, a wait that ran out) are recorded in a device status
+ *    word that moegps_status reads; the kernels skip the offending access instead of faulting.
+ *  - Weight layouts are "output features x input features", so both GEMM operands are contiguous
+ *    along the contraction.
+ */
+#ifndef MOEGPS_H_
+#define MOEGPS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define MOEGPS_API __attribute__((visibility("default")))
+#else
+#define MOEGPS_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum moegps_error {
+  MOEGPS_OK = 0,
+  MOEGPS_ERR_INVALID_ARG = -1,         /* null or misaligned pointer, n_slots != S, bad enum value   */
+  MOEGPS_ERR_UNSUPPORTED_SHAPE = -2,   /* a dimension outside the limits listed at moegps_shape_t    */
+  MOEGPS_ERR_WORKSPACE_TOO_SMALL = -3,
+  MOEGPS_ERR_CUDA = -4,                /* a CUDA runtime/driver call failed (see moegps_last_cuda_error) */
+  MOEGPS_ERR_UNIMPLEMENTED = -5,
+  MOEGPS_ERR_BAD_INDEX = -6,           /* device: an expert/row index outside its range was skipped  */
+  MOEGPS_ERR_TIMEOUT = -7,             /* device: a bounded wait inside a kernel ran out             */
+  MOEGPS_ERR_HIST_MISMATCH = -8        /* device: `hist` passed to dispatch disagrees with topk_idx  */
+} moegps_error;
+
+/* Problem shape, fixed for the life of a context.
+ * Limits: 1 <= K <= min(E, 8); E <= 256; E <= S <= 1024; D and F multiples of 8;
+ * T*K + S*(row_align-1) < 2^31; row_align a power of two in [1, 256]. */
+typedef struct moegps_shape {
+  int32_t T, D, F, E, K, S;
+  int32_t gate_mode;   /* 0: softmax over the K selected logits; 1: sigmoid, then renormalise over the K */
+  int32_t row_align;   /* A: every slot's first row is a multiple of A                                  */
+  int32_t c_max;       /* Algorithm 1's C_max (most copies of one expert); 0 = no cap                   */
+} moegps_shape_t;
+
+typedef struct moegps_ctx moegps_ctx_t;   /* opaque: shape, device id, device status word, cached TMA descriptors */
+
+/* Create / destroy a context on CUDA device `device`.  Allocates the (16-byte) device status word;
+ * this is the only device allocation the library ever makes. */
+MOEGPS_API int moegps_create(moegps_ctx_t** out, const moegps_shape_t* shape, int device);
+MOEGPS_API int moegps_destroy(moegps_ctx_t* ctx);
+
+/* Number of permuted rows Rcap = T*K + S*(row_align-1) the caller must provide for xp/h_ws/yp/row_pair. */
+MOEGPS_API int64_t moegps_rcap(const moegps_shape_t* shape);
+
+/* Bytes of scratch (`workspace`, device, 16-byte aligned) moegps_dispatch needs for this shape. */
+MOEGPS_API size_t moegps_workspace_bytes(const moegps_shape_t* shape);
+
+/* route - top-K gating (paper, Section 2: each token goes to its top-K experts; the mapping is
+ * never altered afterwards).
+ *   logit[t,e] = sum_d x[t,d]*w_router[e,d] + bias[e]   (bf16 inputs, fp32 accumulation)
+ *   topk_idx[t,0..K) = the K experts with the largest logits, in descending logit order; equal
+ *   logits are ordered by ascending expert index.
+ *   topk_w[t,j] = gate weight over the selected K (see moegps_shape_t.gate_mode), fp32.
+ * x: bf16 [T,D]; w_router: bf16 [E,D]; bias: fp32 [E] or NULL; topk_idx: int32 [T,K]; topk_w: fp32 [T,K]. */
+MOEGPS_API int moegps_route(moegps_ctx_t* ctx, const void* x, const void* w_router, const float* bias,
+                 int32_t* topk_idx, float* topk_w, void* stream);
+
+/* Debug companion of moegps_route: also stores the fp32 logits (fp32 [T,E]) the selection was made on. */
+MOEGPS_API int moegps_route_logits(moegps_ctx_t* ctx, const void* x, const void* w_router, const float* bias,
+                        float* logits, void* stream);
+
+/* histogram - per-expert counts n_e of the routed pairs (paper, Eq. 1: p_e = n_e / N with
+ * N = T*K; this is the distribution that Distribution-Only Prediction estimates).
+ * topk_idx: int32 [T*K]; hist: int32 [E].  An index outside [0,E) is skipped and reported as
+ * MOEGPS_ERR_BAD_INDEX through the status word. */
+MOEGPS_API int moegps_histogram(moegps_ctx_t* ctx, const int32_t* topk_idx, int32_t* hist, void* stream);
+
+/* plan - expert duplication from a predicted histogram (paper, Algorithm 1, with one replica per
+ * logical slot and only predicted proportions known, Section 3.2.1): every expert keeps one slot;
+ * each of the S-E extra slots goes to the expert with the largest predicted load per replica
+ * (exact integer comparison; equal ratios go to the fewer replicas, then the lower index) among
+ * experts with fewer than c_max copies.
+ * predicted_hist: int32 [E], >= 0; n_slots must equal shape.S.
+ * replicas: int32 [E]; slot_off: int32 [E+1] (expert e owns slots slot_off[e]..slot_off[e+1]-1);
+ * slot_expert: int32 [S] (-1 for a slot left empty by c_max); bound: int32 [1] = max_e ceil(n_e/r_e). */
+MOEGPS_API int moegps_plan(moegps_ctx_t* ctx, const int32_t* predicted_hist, int32_t n_slots,
+                int32_t* replicas, int32_t* slot_off, int32_t* slot_expert, int32_t* bound, void* stream);
+
+/* dispatch - the routing shuffle (paper, Section 2 all-to-all; Algorithm 1's dispatch d and its
+ * "first tokens" rule): pairs of expert e, in flat pair order, are split into r_e contiguous
+ * balanced ranges (replica rho takes stable ranks floor(rho*n_e/r_e) .. floor((rho+1)*n_e/r_e)-1)
+ * and token rows are copied into the slot buckets in that order.  Lossless: no capacity, no drops.
+ * x: bf16 [T,D]; topk_idx: int32 [T,K]; hist: int32 [E] (actual counts of topk_idx);
+ * replicas, slot_off: from moegps_plan.
+ * slot_row_off: int32 [S+1], slot s owns rows slot_row_off[s]..slot_row_off[s+1]-1, starts are
+ *   multiples of row_align; row_pair: int32 [Rcap] (flat pair of each occupied row, -1 on padding);
+ * pair_row: int32 [T,K]; xp: bf16 [Rcap,D] (padding rows are not written).
+ * workspace: moegps_workspace_bytes(shape) bytes of scratch, contents irrelevant. */
+MOEGPS_API int moegps_dispatch(moegps_ctx_t* ctx, const void* x, const int32_t* topk_idx, const int32_t* hist,
+                    const int32_t* replicas, const int32_t* slot_off,
+                    int32_t* slot_row_off, int32_t* row_pair, int32_t* pair_row,
+                    void* xp, void* workspace, void* stream);
+
+/* expert_ffn - the expert-parallel SwiGLU FFN (paper, Sections 2 and 3.4) over ragged slots:
+ * for every row rho of slot s with e = slot_expert[s]:
+ *   h = silu(w_gate[e] xp[rho]) * (w_up[e] xp[rho]);   yp[rho] = w_down[e] h
+ * bf16 inputs, fp32 accumulation in tensor memory, h and yp rounded to bf16 (nearest even).
+ * xp: bf16 [Rcap,D]; slot_row_off: int32 [S+1]; slot_expert: int32 [S];
+ * w_gate, w_up: bf16 [E,F,D]; w_down: bf16 [E,D,F]; h_ws: bf16 [Rcap,F] scratch; yp: bf16 [Rcap,D].
+ * All rows of a slot's extent are computed (padding rows yield unspecified values); rows outside
+ * every slot and slots with slot_expert < 0 are not written. */
+MOEGPS_API int moegps_expert_ffn(moegps_ctx_t* ctx, const void* xp, const int32_t* slot_row_off,
+                      const int32_t* slot_expert, const void* w_gate, const void* w_up,
+                      const void* w_down, void* h_ws, void* yp, void* stream);
+
+/* The two halves of moegps_expert_ffn as separate calls (same arguments, same kernels), for callers
+ * that want to time or schedule them apart: gate_up writes h_ws = silu(xp w_gate^T) * (xp w_up^T),
+ * down writes yp = h_ws w_down^T.  moegps_expert_ffn is exactly gate_up followed by down. */
+MOEGPS_API int moegps_expert_ffn_gate_up(moegps_ctx_t* ctx, const void* xp, const int32_t* slot_row_off,
+                              const int32_t* slot_expert, const void* w_gate, const void* w_up,
+                              void* h_ws, void* stream);
+MOEGPS_API int moegps_expert_ffn_down(moegps_ctx_t* ctx, const void* h_ws, const int32_t* slot_row_off,
+                           const int32_t* slot_expert, const void* w_down, void* yp, void* stream);
+
+/* combine - the post-FFN shuffle back to token order (paper, Section 2: the same amount of traffic
+ * as the routing shuffle):  out[t,:] = sum_{j<K} topk_w[t,j] * yp[pair_row[t,j],:], fp32
+ * accumulation in ascending j, bf16 result (nearest even).
+ * yp: bf16 [Rcap,D]; pair_row: int32 [T,K]; topk_w: fp32 [T,K]; out: bf16 [T,D]. */
+MOEGPS_API int moegps_combine(moegps_ctx_t* ctx, const void* yp, const int32_t* pair_row, const float* topk_w,
+                   void* out, void* stream);
+
+/* Synchronises `stream`, copies the device status word to *host_status (0 = no device-side error,
+ * else the first moegps_error recorded) and clears it.  Returns MOEGPS_OK or MOEGPS_ERR_CUDA. */
+MOEGPS_API int moegps_status(moegps_ctx_t* ctx, void* stream, int32_t* host_status);
+
+/* Number of kernels this context has launched so far (host-side counter). */
+MOEGPS_API int64_t moegps_launch_count(const moegps_ctx_t* ctx);
+
+/* The cudaError_t (as int) of the last failing CUDA call seen by this context, 0 if none. */
+MOEGPS_API int moegps_last_cuda_error(const moegps_ctx_t* ctx);
+
+MOEGPS_API const char* moegps_error_string(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* MOEGPS_H_ */

@@ -270,7 +270,8 @@ def expert_ffn(xp, slot_row_off, slot_expert, w_gate, w_up, w_down, rows=None) -
     """For every row rho of slot s (expert e = slot_expert[s]):
          g = W1[e] xp[rho],  u = W3[e] xp[rho],  h = silu(g) * u,  Yp[rho] = W2[e] h,
        silu(z) = z / (1 + exp(-z));  no bias terms;  nothing is rounded.
-    W1, W3 are [E, F, D] and W2 is [E, D, F] (output features x input features).
+    W1, W3 are [E, F, D] and W2 is [E, D, F] (output features x input features); they are only
+    ever indexed by expert, so any container with w[e] -> 2-D array will do.
     All rows of a slot's extent [slot_row_off[s], slot_row_off[s+1]) are computed; `rows`
     restricts the work to the listed rows (others stay 0).  Returns Yp fp64 [Rcap, D]."""
     off = [int(v) for v in np.asarray(slot_row_off).reshape(-1)]
@@ -278,8 +279,7 @@ def expert_ffn(xp, slot_row_off, slot_expert, w_gate, w_up, w_down, rows=None) -
     S = len(se)
     xp = np.asarray(xp)
     Rcap = xp.shape[0]
-    Dm = np.asarray(w_down).shape[1]
-    yp = np.zeros((Rcap, Dm), dtype=np.float64)
+    yp = np.zeros((Rcap, xp.shape[1]), dtype=np.float64)      # the FFN maps D back to D
     want = None if rows is None else np.unique(np.asarray(rows, dtype=np.int64))
     for s in range(S):
         e = se[s]

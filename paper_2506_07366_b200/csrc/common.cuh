@@ -1,0 +1,83 @@
+// Shared host/device declarations of the moegps library (context, status word, launch helpers).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "moegps.h"
+
+// Layout of the device status word: [0] first error code, [1] detail (index / location), [2..3] spare.
+struct moegps_ctx {
+  moegps_shape_t shape;
+  int device;
+  int sm_count;
+  int32_t* d_status;        // 4 x int32 on the device
+  int64_t launches;         // kernels launched through this context
+  int last_cuda_error;
+  // cached TMA descriptors of the expert FFN, keyed by the base pointers they were built for
+  const void* tm_key1[3];   // xp, w_gate, w_up
+  CUtensorMap tm_xp, tm_w1, tm_w3;
+  bool tm1_valid;
+  const void* tm_key2[2];   // h_ws, w_down
+  CUtensorMap tm_h, tm_w2;
+  bool tm2_valid;
+  bool ffn_attr_done;    // dynamic shared-memory limit of the GEMM kernels raised on this device
+  // cached TMA descriptors of the router
+  const void* rt_key[2];
+  CUtensorMap tm_rx, tm_rw;
+  bool rt_valid;
+};
+
+#define MOEGPS_CUDA_TRY(ctx, expr)                                   \
+  do {                                                               \
+    cudaError_t _e = (expr);                                         \
+    if (_e != cudaSuccess) {                                         \
+      (ctx)->last_cuda_error = (int)_e;                              \
+      return MOEGPS_ERR_CUDA;                                        \
+    }                                                                \
+  } while (0)
+
+// Records a launch (and its launch error, if any).
+#define MOEGPS_AFTER_LAUNCH(ctx)                                     \
+  do {                                                               \
+    (ctx)->launches += 1;                                            \
+    cudaError_t _e = cudaGetLastError();                             \
+    if (_e != cudaSuccess) {                                         \
+      (ctx)->last_cuda_error = (int)_e;                              \
+      return MOEGPS_ERR_CUDA;                                        \
+    }                                                                \
+  } while (0)
+
+static inline bool moegps_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static inline int64_t moegps_rcap_of(const moegps_shape_t& s) {
+  return (int64_t)s.T * s.K + (int64_t)s.S * (s.row_align - 1);
+}
+
+// First error wins; later ones are dropped.
+__device__ __forceinline__ void moegps_report(int32_t* status, int code, int detail) {
+  if (atomicCAS(&status[0], 0, code) == 0) status[1] = detail;
+}
+
+// dispatch: pairs per warp segment of the stable ranking (see dispatch.cu)
+constexpr int kSegPairs = 256;
+
+// Per-step launchers (each validates nothing: the C entry points in api.cu do that).
+int moegps_launch_route(moegps_ctx* ctx, const void* x, const void* wr, const float* bias,
+                        int32_t* topk_idx, float* topk_w, float* logits_out, cudaStream_t st);
+int moegps_launch_histogram(moegps_ctx* ctx, const int32_t* topk_idx, int32_t* hist, cudaStream_t st);
+int moegps_launch_plan(moegps_ctx* ctx, const int32_t* pred, int32_t* replicas, int32_t* slot_off,
+                       int32_t* slot_expert, int32_t* bound, cudaStream_t st);
+int moegps_launch_dispatch(moegps_ctx* ctx, const void* x, const int32_t* topk_idx, const int32_t* hist,
+                           const int32_t* replicas, const int32_t* slot_off, int32_t* slot_row_off,
+                           int32_t* row_pair, int32_t* pair_row, void* xp, void* workspace,
+                           cudaStream_t st);
+int moegps_launch_ffn_gate_up(moegps_ctx* ctx, const void* xp, const int32_t* slot_row_off,
+                              const int32_t* slot_expert, const void* w_gate, const void* w_up, void* h_ws,
+                              cudaStream_t st);
+int moegps_launch_ffn_down(moegps_ctx* ctx, const void* h_ws, const int32_t* slot_row_off,
+                           const int32_t* slot_expert, const void* w_down, void* yp, cudaStream_t st);
+int moegps_launch_combine(moegps_ctx* ctx, const void* yp, const int32_t* pair_row, const float* topk_w,
+                          void* out, cudaStream_t st);

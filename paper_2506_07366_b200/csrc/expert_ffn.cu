@@ -1,0 +1,364 @@
+// expert_ffn: the expert-parallel SwiGLU FFN (paper, Sections 2 and 3.4) over ragged slots, as two
+// persistent grouped GEMMs on the 5th-generation tensor cores:
+//   GEMM 1:  H  = silu(Xp W1[e]^T) * (Xp W3[e]^T)      (gate and up share the A tile; SwiGLU epilogue)
+//   GEMM 2:  Yp = H W2[e]^T
+// Tile = 128 rows of one slot x 256 accumulator columns (GEMM 1: 128 gate + 128 up columns).
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (one elected thread; owns TMEM),
+// warps 2..5 = epilogue (each reads its quarter of the 128 TMEM lanes).  A 4-stage shared-memory ring
+// (TMA -> tcgen05.mma) and two TMEM accumulators (mainloop of tile i+1 overlaps the epilogue of tile
+// i) are handed around with mbarriers; every wait is bounded and raises an abort flag on expiry.
+// Tiles are enumerated on the device from slot_row_off (no host round trip): slot-major, then
+// column tile, then row tile, so that CTAs working at the same time share weight tiles in L2.
+#include "common.cuh"
+#include "sm100.cuh"
+
+namespace {
+
+using namespace sm100;
+
+constexpr int BM = 128;            // rows per tile
+constexpr int BNACC = 256;         // accumulator columns per tile
+constexpr int BK = 64;             // K elements per stage: 128 bytes = one swizzle row
+constexpr int kStages = 4;
+constexpr int kABytes = BM * BK * 2;
+constexpr int kBHalfBytes = 128 * BK * 2;
+constexpr int kStageBytes = kABytes + 2 * kBHalfBytes;       // 48 KiB
+constexpr int kThreads = 192;
+constexpr int kMaxS = 1024;
+constexpr int kTmemCols = 512;
+
+struct __align__(16) Tables {
+  int32_t tile_base[kMaxS + 1];    // first tile index of each slot
+  int32_t row_off[kMaxS + 1];
+  int32_t expert[kMaxS];
+};
+
+constexpr size_t kSmemBytes = 1024 /* alignment slack */ + (size_t)kStages * kStageBytes + sizeof(Tables) + 256;
+
+struct TileCoord {
+  int m0;        // first row of the tile in the permuted buffer
+  int row_end;   // one past the last row of the slot's extent
+  int n_tile;
+  int expert;
+};
+
+__device__ __forceinline__ TileCoord decode_tile(const Tables& tb, int S, int tile, int n_tiles) {
+  int lo = 0, hi = S;                 // find s with tile_base[s] <= tile < tile_base[s+1]
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (tb.tile_base[mid] <= tile) lo = mid; else hi = mid;
+  }
+  const int s = lo;
+  const int local = tile - tb.tile_base[s];
+  const int mt = (tb.tile_base[s + 1] - tb.tile_base[s]) / n_tiles;   // row tiles of this slot
+  TileCoord c;
+  c.n_tile = local / mt;
+  c.m0 = tb.row_off[s] + (local % mt) * BM;
+  c.row_end = tb.row_off[s + 1];
+  c.expert = tb.expert[s];
+  return c;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+// kSwiGLU = true : out[row, n_tile*128 + c] = silu(acc[c]) * acc[128 + c],  c < 128
+// kSwiGLU = false: out[row, n_tile*256 + c] = acc[c],                        c < 256
+template <bool kSwiGLU>
+__global__ void __launch_bounds__(kThreads, 1)
+grouped_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
+                    const __grid_constant__ CUtensorMap tm_b1, const int32_t* __restrict__ slot_row_off,
+                    const int32_t* __restrict__ slot_expert, int S, int E, int n_dim, int k_dim,
+                    __nv_bfloat16* __restrict__ out, int32_t* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* stage_mem = smem;                                          // kStages x (A | B0 | B1), 1024-aligned
+  Tables& tb = *reinterpret_cast<Tables*>(smem + (size_t)kStages * kStageBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kStages * kStageBytes + sizeof(Tables));
+  uint64_t* full = bars;                  // [kStages]  TMA -> MMA
+  uint64_t* empty = bars + kStages;       // [kStages]  MMA -> TMA
+  uint64_t* acc_full = bars + 2 * kStages;       // [2]  MMA -> epilogue
+  uint64_t* acc_empty = bars + 2 * kStages + 2;  // [2]  epilogue -> MMA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  int* total_tiles_p = const_cast<int*>(reinterpret_cast<volatile int*>(tmem_slot + 2));
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int cols_per_tile = kSwiGLU ? 128 : 256;
+  const int n_tiles = (n_dim + cols_per_tile - 1) / cols_per_tile;
+  const int num_kb = (k_dim + BK - 1) / BK;
+
+  // ---------------------------------------------------------------- set-up
+  for (int s = threadIdx.x; s <= S; s += kThreads) tb.row_off[s] = slot_row_off[s];
+  for (int s = threadIdx.x; s < S; s += kThreads) tb.expert[s] = slot_expert[s];
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 4); }
+    *abort_flag = 0;
+    fence_mbar_init();
+    prefetch_tensormap(&tm_a);
+    prefetch_tensormap(&tm_b0);
+    prefetch_tensormap(&tm_b1);
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, kTmemCols);
+    tmem_relinquish();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int acc = 0;
+    for (int s = 0; s < S; ++s) {
+      tb.tile_base[s] = acc;
+      const int rows = tb.row_off[s + 1] - tb.row_off[s];
+      const int e = tb.expert[s];
+      if (rows > 0 && e >= 0 && e < E) acc += ((rows + BM - 1) / BM) * n_tiles;
+      else if (rows > 0 && e >= E) moegps_report(status, MOEGPS_ERR_BAD_INDEX, s);
+    }
+    tb.tile_base[S] = acc;
+    *total_tiles_p = acc;
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  const int total_tiles = *total_tiles_p;
+
+  // ---------------------------------------------------------------- roles
+  if (warp == 0) {
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+        const TileCoord tc = decode_tile(tb, S, tile, n_tiles);
+        const int nb0 = tc.n_tile * cols_per_tile;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
+          uint8_t* sa = stage_mem + (size_t)stage * kStageBytes;
+          mbar_arrive_expect_tx(&full[stage], kStageBytes);
+          tma_load_2d(sa, &tm_a, &full[stage], kb * BK, tc.m0);
+          tma_load_3d(sa + kABytes, &tm_b0, &full[stage], kb * BK, nb0, tc.expert);
+          tma_load_3d(sa + kABytes + kBHalfBytes, &tm_b1, &full[stage], kb * BK, kSwiGLU ? nb0 : nb0 + 128,
+                      tc.expert);
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // let copies that are still in flight land before the CTA retires
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = idesc_bf16_f32(BM, BNACC);
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+        if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + (uint32_t)acc * BNACC;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
+          tc_fence_after_sync();
+          const uint32_t sa = smem_u32(stage_mem + (size_t)stage * kStageBytes);
+          const uint64_t da = smem_desc_k_sw128(sa);
+          const uint64_t db = smem_desc_k_sw128(sa + kABytes);
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k)      // 16 bf16 = 32 bytes per MMA along K
+            mma_bf16(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb | k) != 0);
+          mma_commit(&empty[stage]);             // frees the stage when these MMAs have read it
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        mma_commit(&acc_full[acc]);              // accumulator complete
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+      if (!ok) {
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+      }
+    }
+  } else {
+    const int quarter = warp & 3;                 // TMEM lanes this warp may read
+    const int row_in_tile = quarter * 32 + lane;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+      const TileCoord tc = decode_tile(tb, S, tile, n_tiles);
+      if (!mbar_wait(&acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
+      tc_fence_after_sync();
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * BNACC;
+      const int row = tc.m0 + row_in_tile;
+      const bool row_ok = row < tc.row_end;
+      const int col0 = tc.n_tile * cols_per_tile;
+      __nv_bfloat16* orow = out + (size_t)row * n_dim + col0;
+      if constexpr (kSwiGLU) {
+#pragma unroll 1
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+          uint32_t g[32], u[32];
+          tmem_ld32(taddr + c0, g);
+          tmem_ld32(taddr + 128 + c0, u);
+          tmem_ld_wait();
+          uint32_t o[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
+            const float h0 = g0 / (1.f + __expf(-g0)) * __uint_as_float(u[2 * i]);
+            const float h1 = g1 / (1.f + __expf(-g1)) * __uint_as_float(u[2 * i + 1]);
+            o[i] = pack_bf16(h0, h1);
+          }
+          if (row_ok) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v)
+              if (col0 + c0 + 8 * v + 8 <= n_dim)
+                *reinterpret_cast<uint4*>(orow + c0 + 8 * v) = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
+          }
+        }
+      } else {
+#pragma unroll 1
+        for (int c0 = 0; c0 < 256; c0 += 32) {
+          uint32_t a[32];
+          tmem_ld32(taddr + c0, a);
+          tmem_ld_wait();
+          uint32_t o[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) o[i] = pack_bf16(__uint_as_float(a[2 * i]), __uint_as_float(a[2 * i + 1]));
+          if (row_ok) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v)
+              if (col0 + c0 + 8 * v + 8 <= n_dim)
+                *reinterpret_cast<uint4*>(orow + c0 + 8 * v) = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
+          }
+        }
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[acc]);
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  // ---------------------------------------------------------------- teardown
+  __syncwarp();
+  tc_fence_before_sync();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) moegps_report(status, MOEGPS_ERR_TIMEOUT, (int)blockIdx.x);
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+}  // namespace
+
+// bf16 [rows, cols] row-major; box = 64 columns x box_rows rows, 128-byte swizzle, zero fill outside.
+bool moegps_make_tmap_2d(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols * 2};
+  const cuuint32_t box[2] = {64, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// bf16 [batch, rows, cols]; box = 64 columns x box_rows rows x 1 batch entry.
+bool moegps_make_tmap_3d(CUtensorMap* tm, const void* base, uint64_t batch, uint64_t rows, uint64_t cols,
+                         uint32_t box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[3] = {cols, rows, batch};
+  const cuuint64_t strides[2] = {cols * 2, rows * cols * 2};
+  const cuuint32_t box[3] = {64, box_rows, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+namespace {
+
+int raise_smem_limit(moegps_ctx* ctx) {
+  if (ctx->ffn_attr_done) return MOEGPS_OK;
+  MOEGPS_CUDA_TRY(ctx, cudaFuncSetAttribute(grouped_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)kSmemBytes));
+  MOEGPS_CUDA_TRY(ctx, cudaFuncSetAttribute(grouped_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)kSmemBytes));
+  ctx->ffn_attr_done = true;
+  return MOEGPS_OK;
+}
+
+int tmap_failed(moegps_ctx* ctx) {
+  ctx->last_cuda_error = (int)cudaErrorInvalidValue;
+  return MOEGPS_ERR_CUDA;
+}
+
+}  // namespace
+
+int moegps_launch_ffn_gate_up(moegps_ctx* ctx, const void* xp, const int32_t* slot_row_off,
+                              const int32_t* slot_expert, const void* w_gate, const void* w_up, void* h_ws,
+                              cudaStream_t st) {
+  const moegps_shape_t& s = ctx->shape;
+  const uint64_t rcap = (uint64_t)moegps_rcap_of(s);
+  if (!(ctx->tm1_valid && ctx->tm_key1[0] == xp && ctx->tm_key1[1] == w_gate && ctx->tm_key1[2] == w_up)) {
+    ctx->tm1_valid = false;
+    if (!(moegps_make_tmap_2d(&ctx->tm_xp, xp, rcap, s.D, BM) &&
+          moegps_make_tmap_3d(&ctx->tm_w1, w_gate, s.E, s.F, s.D, 128) &&
+          moegps_make_tmap_3d(&ctx->tm_w3, w_up, s.E, s.F, s.D, 128)))
+      return tmap_failed(ctx);
+    ctx->tm_key1[0] = xp; ctx->tm_key1[1] = w_gate; ctx->tm_key1[2] = w_up;
+    ctx->tm1_valid = true;
+  }
+  int rc = raise_smem_limit(ctx);
+  if (rc != MOEGPS_OK) return rc;
+  grouped_gemm_kernel<true><<<ctx->sm_count, kThreads, kSmemBytes, st>>>(
+      ctx->tm_xp, ctx->tm_w1, ctx->tm_w3, slot_row_off, slot_expert, s.S, s.E, s.F, s.D,
+      static_cast<__nv_bfloat16*>(h_ws), ctx->d_status);
+  MOEGPS_AFTER_LAUNCH(ctx);
+  return MOEGPS_OK;
+}
+
+int moegps_launch_ffn_down(moegps_ctx* ctx, const void* h_ws, const int32_t* slot_row_off,
+                           const int32_t* slot_expert, const void* w_down, void* yp, cudaStream_t st) {
+  const moegps_shape_t& s = ctx->shape;
+  const uint64_t rcap = (uint64_t)moegps_rcap_of(s);
+  if (!(ctx->tm2_valid && ctx->tm_key2[0] == h_ws && ctx->tm_key2[1] == w_down)) {
+    ctx->tm2_valid = false;
+    if (!(moegps_make_tmap_2d(&ctx->tm_h, h_ws, rcap, s.F, BM) &&
+          moegps_make_tmap_3d(&ctx->tm_w2, w_down, s.E, s.D, s.F, 128)))
+      return tmap_failed(ctx);
+    ctx->tm_key2[0] = h_ws; ctx->tm_key2[1] = w_down;
+    ctx->tm2_valid = true;
+  }
+  int rc = raise_smem_limit(ctx);
+  if (rc != MOEGPS_OK) return rc;
+  grouped_gemm_kernel<false><<<ctx->sm_count, kThreads, kSmemBytes, st>>>(
+      ctx->tm_h, ctx->tm_w2, ctx->tm_w2, slot_row_off, slot_expert, s.S, s.E, s.D, s.F,
+      static_cast<__nv_bfloat16*>(yp), ctx->d_status);
+  MOEGPS_AFTER_LAUNCH(ctx);
+  return MOEGPS_OK;
+}

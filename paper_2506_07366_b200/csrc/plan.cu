@@ -1,0 +1,124 @@
+// plan: Algorithm 1 of the paper in slot form, on one CTA.  Thread e keeps (n_e, r_e) in registers;
+// each of the S-E rounds is a block-wide arg-max of n_e / r_e (exact: 64-bit cross-multiplication)
+// that hands the next free slot to the winner.  Integer only.
+#include "common.cuh"
+
+namespace {
+
+constexpr int kPlanThreads = 256;   // >= the largest supported E
+
+struct Cand {
+  long long n;   // predicted count; -1 marks "not eligible"
+  int r;
+  int e;
+};
+
+// Strict order of Algorithm 1's choice: larger n/r first, then fewer replicas, then lower index.
+__device__ __forceinline__ bool better(const Cand& a, const Cand& b) {
+  if (a.n < 0) return false;
+  if (b.n < 0) return true;
+  const long long lhs = a.n * (long long)b.r;
+  const long long rhs = b.n * (long long)a.r;
+  if (lhs != rhs) return lhs > rhs;
+  if (a.r != b.r) return a.r < b.r;
+  return a.e < b.e;
+}
+
+__device__ __forceinline__ Cand shfl_xor(const Cand& c, int m) {
+  Cand o;
+  o.n = __shfl_xor_sync(0xffffffffu, c.n, m);
+  o.r = __shfl_xor_sync(0xffffffffu, c.r, m);
+  o.e = __shfl_xor_sync(0xffffffffu, c.e, m);
+  return o;
+}
+
+__device__ __forceinline__ Cand warp_best(Cand c) {
+#pragma unroll
+  for (int m = 16; m >= 1; m >>= 1) {
+    const Cand o = shfl_xor(c, m);
+    if (better(o, c)) c = o;
+  }
+  return c;
+}
+
+__global__ void __launch_bounds__(kPlanThreads)
+plan_kernel(const int32_t* __restrict__ pred, int E, int S, int c_max, int32_t* __restrict__ replicas,
+            int32_t* __restrict__ slot_off, int32_t* __restrict__ slot_expert, int32_t* __restrict__ bound,
+            int32_t* __restrict__ status) {
+  __shared__ Cand warp_c[kPlanThreads / 32];
+  __shared__ Cand winner;
+  __shared__ int warp_sum[kPlanThreads / 32];
+  __shared__ int warp_max[kPlanThreads / 32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const bool mine = tid < E;
+  long long n = -1;
+  int r = 0;
+  if (mine) {
+    const int v = pred[tid];
+    if (v < 0) moegps_report(status, MOEGPS_ERR_BAD_INDEX, tid);
+    n = v < 0 ? 0 : v;
+    r = 1;
+  }
+  for (int round = 0; round < S - E; ++round) {
+    Cand c;
+    c.n = (mine && (c_max <= 0 || r < c_max)) ? n : -1;
+    c.r = r;
+    c.e = tid;
+    c = warp_best(c);
+    if (lane == 0) warp_c[warp] = c;
+    __syncthreads();
+    if (warp == 0) {
+      Cand d;
+      d.n = -1; d.r = 0; d.e = kPlanThreads + lane;
+      if (lane < kPlanThreads / 32) d = warp_c[lane];
+      d = warp_best(d);
+      if (lane == 0) winner = d;
+    }
+    __syncthreads();
+    const Cand w = winner;
+    if (w.n < 0) break;            // nobody may take another copy: the remaining slots stay empty
+    if (w.e == tid) r += 1;
+    // `winner`/`warp_c` are rewritten only after the next round's first barrier
+  }
+  // slot_off = exclusive prefix sum of r
+  int incl = mine ? r : 0;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const int o = __shfl_up_sync(0xffffffffu, incl, d);
+    if (lane >= d) incl += o;
+  }
+  if (lane == 31) warp_sum[warp] = incl;
+  int b = mine ? (int)((n + r - 1) / r) : 0;     // ceil(n_e / r_e)
+#pragma unroll
+  for (int m = 16; m >= 1; m >>= 1) b = max(b, __shfl_xor_sync(0xffffffffu, b, m));
+  if (lane == 0) warp_max[warp] = b;
+  __syncthreads();
+  int base = 0, total = 0, bmax = 0;
+  for (int wv = 0; wv < kPlanThreads / 32; ++wv) {
+    if (wv < warp) base += warp_sum[wv];
+    total += warp_sum[wv];
+    bmax = max(bmax, warp_max[wv]);
+  }
+  const int excl = base + incl - (mine ? r : 0);
+  if (mine) {
+    replicas[tid] = r;
+    slot_off[tid] = excl;
+    for (int s = excl; s < excl + r; ++s) slot_expert[s] = tid;
+  }
+  if (tid == 0) {
+    slot_off[E] = total;
+    bound[0] = bmax;
+  }
+  for (int s = total + tid; s < S; s += kPlanThreads) slot_expert[s] = -1;
+}
+
+}  // namespace
+
+int moegps_launch_plan(moegps_ctx* ctx, const int32_t* pred, int32_t* replicas, int32_t* slot_off,
+                       int32_t* slot_expert, int32_t* bound, cudaStream_t st) {
+  const moegps_shape_t& s = ctx->shape;
+  plan_kernel<<<1, kPlanThreads, 0, st>>>(pred, s.E, s.S, s.c_max, replicas, slot_off, slot_expert, bound,
+                                          ctx->d_status);
+  MOEGPS_AFTER_LAUNCH(ctx);
+  return MOEGPS_OK;
+}

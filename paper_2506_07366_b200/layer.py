@@ -1,0 +1,67 @@
+"""One MoE layer with prediction-driven expert duplication, driven through the C ABI.
+
+`MoeLayer` owns the device buffers (allocated once with torch) and chains the six library calls on
+the current stream; no step runs anywhere but in the library's kernels.
+"""
+from __future__ import annotations
+
+import torch
+
+from .binding import Context, Shape, workspace_bytes
+
+
+class MoeLayer:
+    def __init__(self, shape: Shape, w_router, bias, w_gate, w_up, w_down, device=None):
+        self.shape = s = shape
+        self.ctx = Context(shape, device)
+        dev = w_router.device
+        self.w_router, self.bias = w_router, bias
+        self.w_gate, self.w_up, self.w_down = w_gate, w_up, w_down
+        i32 = dict(dtype=torch.int32, device=dev)
+        bf = dict(dtype=torch.bfloat16, device=dev)
+        self.x = torch.empty(s.T, s.D, **bf)             # staging for host inputs
+        self.topk_idx = torch.empty(s.T, s.K, **i32)
+        self.topk_w = torch.empty(s.T, s.K, dtype=torch.float32, device=dev)
+        self.hist = torch.empty(s.E, **i32)
+        self.replicas = torch.empty(s.E, **i32)
+        self.slot_off = torch.empty(s.E + 1, **i32)
+        self.slot_expert = torch.empty(s.S, **i32)
+        self.bound = torch.empty(1, **i32)
+        self.slot_row_off = torch.empty(s.S + 1, **i32)
+        self.row_pair = torch.empty(s.Rcap, **i32)
+        self.pair_row = torch.empty(s.T, s.K, **i32)
+        self.xp = torch.empty(s.Rcap, s.D, **bf)
+        self.h_ws = torch.empty(s.Rcap, s.F, **bf)
+        self.yp = torch.empty(s.Rcap, s.D, **bf)
+        self.out = torch.empty(s.T, s.D, **bf)
+        self.workspace = torch.empty(max(16, workspace_bytes(s)), dtype=torch.uint8, device=dev)
+        self.pred = torch.empty(s.E, **i32)
+        self._planned = False
+
+    def plan(self, predicted_hist, stream=None):
+        """Replica plan from a predicted histogram (int32 [E], device or host tensor)."""
+        self.pred.copy_(predicted_hist.to(torch.int32), non_blocking=True)
+        self.ctx.plan(self.pred, self.shape.S, self.replicas, self.slot_off, self.slot_expert,
+                      self.bound, stream)
+        self._planned = True
+
+    def forward(self, x, stream=None):
+        """route -> histogram -> dispatch -> expert_ffn -> combine on device tensor x [T, D]."""
+        if not self._planned:
+            raise RuntimeError("call plan(predicted_hist) before forward()")
+        c = self.ctx
+        c.route(x, self.w_router, self.bias, self.topk_idx, self.topk_w, stream)
+        c.histogram(self.topk_idx, self.hist, stream)
+        c.dispatch(x, self.topk_idx, self.hist, self.replicas, self.slot_off, self.slot_row_off,
+                   self.row_pair, self.pair_row, self.xp, self.workspace, stream)
+        c.expert_ffn(self.xp, self.slot_row_off, self.slot_expert, self.w_gate, self.w_up,
+                     self.w_down, self.h_ws, self.yp, stream)
+        c.combine(self.yp, self.pair_row, self.topk_w, self.out, stream)
+        return self.out
+
+    def forward_host(self, x_host, out_host, stream=None):
+        """Same, with (pinned) host tensors: copies x in, runs the layer, copies the result out."""
+        self.x.copy_(x_host, non_blocking=True)
+        out = self.forward(self.x, stream)
+        out_host.copy_(out, non_blocking=True)
+        return out_host

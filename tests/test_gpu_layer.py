@@ -1,0 +1,153 @@
+"""Whole-layer parity: MoeLayer (route -> histogram -> plan -> dispatch -> expert_ffn -> combine
+through the C ABI) against the oracle.
+
+Small and scaled-down workloads are compared element by element.  The full-size workloads are run
+in the launch configuration the benchmark times; their integer steps are compared exactly over the
+whole batch and their float outputs on sampled tokens the oracle computes one by one.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2506_07366_b200 import binding, workloads as wl
+from paper_2506_07366_b200.layer import MoeLayer
+from tests import harness as hz
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+SMALL = [
+    (wl.WORKLOADS["tiny"], 128),
+    (wl.WORKLOADS["tiny"], 1),
+    (wl.WORKLOADS["mixtral"].scaled(T=384, D=512, F=1792), 128),
+    (wl.WORKLOADS["mixtral_skew"].scaled(T=1024, D=256, F=896), 128),
+    (wl.WORKLOADS["many_expert"].scaled(T=512, D=256, F=352), 128),
+    (wl.WORKLOADS["fine_grained"].scaled(T=256, D=448, F=128), 128),
+    (wl.WORKLOADS["fine_grained"].scaled(T=256, D=448, F=128), 16),
+]
+
+
+def build_inputs(w, device):
+    wr, bias = wl.router(w, "cpu")
+    x, _ = hz.screened_activations(w, wr, bias)
+    w1, w3, w2 = wl.expert_weights(w, "cpu")
+    return x, wr, bias, w1, w3, w2
+
+
+@pytest.mark.parametrize("w,A", SMALL, ids=lambda v: v if isinstance(v, int) else f"{v.name}-T{v.T}")
+def test_layer_small(w, A):
+    x, wr, bias, w1, w3, w2 = build_inputs(w, DEV)
+    ref_idx, _, _ = oracle.route(hz.bits(x), hz.bits(wr), bias.numpy(), w.K, w.gate_mode)
+    pred = hz.predicted_histogram(w, oracle.histogram(ref_idx, w.E), wr, bias)
+    ref = oracle.moe_layer(hz.bits(x), hz.bits(wr), bias.numpy(), hz.bits(w1), hz.bits(w3), hz.bits(w2), pred,
+                           K=w.K, S=w.S, gate_mode=w.gate_mode, row_align=A)
+    shape = binding.Shape(w.T, w.D, w.F, w.E, w.K, w.S, w.gate_mode, A)
+    layer = MoeLayer(shape, wr.to(DEV), bias.to(DEV), w1.to(DEV), w3.to(DEV), w2.to(DEV))
+    layer.out.fill_(float("nan"))
+    layer.plan(torch.from_numpy(pred))
+    out = layer.forward(x.to(DEV))
+    layer.ctx.check_status()
+    for name in ("replicas", "slot_off", "slot_expert", "topk_idx", "hist", "slot_row_off", "row_pair", "pair_row"):
+        assert np.array_equal(getattr(layer, name).cpu().numpy(), ref[name]), name
+    assert int(layer.bound.item()) == ref["bound"]
+    hz.assert_close_rel_max(layer.topk_w.cpu().numpy(), ref["topk_w"], "topk_w")
+    occ = ref["row_pair"] >= 0
+    assert np.array_equal(hz.bits(layer.xp)[occ], ref["xp"][occ])
+    hz.assert_close_rel_max(layer.yp.float().cpu().numpy()[occ], ref["yp"][occ], "yp")
+    hz.assert_close_rel_max(out.float().cpu().numpy(), ref["out"], "out")
+    # placement never changes results: same layer without duplication (S = E), compact rows
+    shape2 = binding.Shape(w.T, w.D, w.F, w.E, w.K, w.E, w.gate_mode, 1)
+    layer2 = MoeLayer(shape2, wr.to(DEV), bias.to(DEV), w1.to(DEV), w3.to(DEV), w2.to(DEV))
+    layer2.plan(torch.zeros(w.E, dtype=torch.int32))
+    out2 = layer2.forward(x.to(DEV))
+    layer2.ctx.check_status()
+    assert torch.equal(out2, out)      # same rows, same arithmetic order => bitwise equal
+
+
+def test_layer_host_buffers():
+    w = wl.WORKLOADS["tiny"]
+    x, wr, bias, w1, w3, w2 = build_inputs(w, DEV)
+    shape = binding.Shape(w.T, w.D, w.F, w.E, w.K, w.S, w.gate_mode, 128)
+    layer = MoeLayer(shape, wr.to(DEV), bias.to(DEV), w1.to(DEV), w3.to(DEV), w2.to(DEV))
+    layer.plan(torch.ones(w.E, dtype=torch.int32))
+    xh = x.pin_memory()
+    oh = torch.empty(w.T, w.D, dtype=torch.bfloat16).pin_memory()
+    layer.forward_host(xh, oh)
+    torch.cuda.synchronize()
+    assert torch.equal(oh, layer.forward(x.to(DEV)).cpu())
+
+
+class ExpertsOnDemand:
+    """w[e] -> host bf16 bits of one expert's matrix, fetched from the device when asked for."""
+
+    def __init__(self, t):
+        self.t = t
+
+    def __getitem__(self, e):
+        return hz.bits(self.t[int(e)])
+
+
+FULL = ["mixtral", "mixtral_skew", "many_expert", "fine_grained"]
+
+
+@pytest.mark.parametrize("name", FULL)
+def test_layer_full_size_sampled(name):
+    w = wl.WORKLOADS[name]
+    torch.cuda.empty_cache()
+    wr, bias = wl.router(w, DEV)
+    x0 = wl.activations(w, DEV)
+    x, redrawn = hz.screened_activations(w, wr.cpu(), bias.cpu(), x0.cpu())
+    assert redrawn <= 0.05 * w.T
+    w1, w3, w2 = wl.expert_weights(w, DEV)
+    xb, wrb, bb = hz.bits(x), hz.bits(wr), bias.cpu().numpy()
+    ref_idx, ref_w, ref_logits = oracle.route(xb, wrb, bb, w.K, w.gate_mode)
+    ref_hist = oracle.histogram(ref_idx, w.E)
+    pred = hz.predicted_histogram(w, ref_hist, wr.cpu(), bias.cpu())
+    A = 128
+    rep, so, se, bound = oracle.plan(pred, w.S)
+    sro, rp, pr, _ = oracle.dispatch(None, ref_idx, ref_hist, rep, so, w.S, A)
+
+    shape = binding.Shape(w.T, w.D, w.F, w.E, w.K, w.S, w.gate_mode, A)
+    layer = MoeLayer(shape, wr, bias, w1, w3, w2)
+    layer.plan(torch.from_numpy(pred))
+    xd = x.to(DEV)
+    out = layer.forward(xd)
+    layer.ctx.check_status()
+    logits = torch.empty(w.T, w.E, dtype=torch.float32, device=DEV)
+    layer.ctx.route_logits(xd, wr, bias, logits)
+    assert np.abs(logits.cpu().numpy().astype(np.float64) - ref_logits).max() < hz.TAU / 4
+
+    # integer steps: exact over the whole batch
+    assert np.array_equal(layer.topk_idx.cpu().numpy(), ref_idx)
+    assert np.array_equal(layer.hist.cpu().numpy(), ref_hist)
+    assert np.array_equal(layer.replicas.cpu().numpy(), rep)
+    assert np.array_equal(layer.slot_off.cpu().numpy(), so)
+    assert np.array_equal(layer.slot_expert.cpu().numpy(), se)
+    assert int(layer.bound.item()) == bound
+    assert np.array_equal(layer.slot_row_off.cpu().numpy(), sro)
+    assert np.array_equal(layer.row_pair.cpu().numpy(), rp)
+    assert np.array_equal(layer.pair_row.cpu().numpy(), pr)
+    hz.assert_close_rel_max(layer.topk_w.cpu().numpy(), ref_w, "topk_w")
+    # properties that hold at any size, checked on the device results
+    assert int(layer.hist.sum()) == w.T * w.K
+    rows = layer.pair_row.reshape(-1).long()
+    assert torch.equal(layer.row_pair[rows].long(), torch.arange(w.R, device=DEV))
+    assert torch.equal(layer.xp[rows], xd.repeat_interleave(w.K, dim=0))       # rows are bit copies
+    loads = np.diff(sro)
+    assert loads.max() <= -(-int(np.ceil(max(1.0, (ref_hist / np.maximum(pred, 1)).max()) * bound)) // A) * A
+
+    # float outputs on sampled tokens (first, last, and a seeded draw, covering hot and cold experts)
+    rng = np.random.default_rng(w.seed)
+    tokens = np.unique(np.concatenate([[0, w.T - 1], rng.choice(w.T, size=10, replace=False)]))
+    sample_rows = pr[tokens].reshape(-1)
+    xp_bits = np.zeros((shape.Rcap, w.D), dtype=np.uint16)
+    xp_bits[sample_rows] = xb[np.repeat(tokens, w.K)]
+    yp_ref = oracle.expert_ffn(xp_bits, sro, se, ExpertsOnDemand(w1), ExpertsOnDemand(w3), ExpertsOnDemand(w2),
+                               rows=sample_rows)
+    out_ref = oracle.combine(yp_ref, pr, ref_w, tokens=tokens)
+    yp_got = layer.yp[torch.from_numpy(sample_rows).to(DEV).long()].float().cpu().numpy()
+    hz.assert_close_rel_max(yp_got, yp_ref[sample_rows], "yp (sampled rows)")
+    out_got = out[torch.from_numpy(tokens).to(DEV).long()].float().cpu().numpy()
+    hz.assert_close_rel_max(out_got, out_ref[tokens], "out (sampled tokens)")
+    assert torch.isfinite(out.float()).all()

@@ -1,0 +1,333 @@
+"""Per-step parity of the CUDA kernels (through the C ABI) with the CPU oracle.
+
+Each step is fed the ORACLE's inputs for that step, so a defect in one kernel cannot hide behind, or
+be blamed on, another.  Integers must match exactly; floats within 2e-2 * max|ref| (tighter where
+the arithmetic allows it).  Outputs are poison-filled before every call so that an unwritten or
+over-written element shows up.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2506_07366_b200 import binding, workloads as wl
+from tests import harness as hz
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def i32(a):
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(DEV)
+
+
+def poison_i32(*shape):
+    return torch.full(shape, -7777, dtype=torch.int32, device=DEV)
+
+
+def poison_bf16(*shape):
+    return torch.full(shape, float("nan"), dtype=torch.bfloat16, device=DEV)
+
+
+def small(name, **kw):
+    return wl.WORKLOADS[name].scaled(**kw)
+
+
+ROUTE_CASES = [
+    wl.WORKLOADS["tiny"],
+    small("mixtral", T=333, D=1024),
+    small("many_expert", T=257, D=512),
+    small("fine_grained", T=130, D=1024),
+    small("fine_grained", T=64, D=256, E=200, K=8, S=200),
+    small("tiny", T=65, D=64, E=5, K=5, S=5),
+    small("tiny", T=40, D=64, E=33, K=1, S=40, gate_mode=1),
+]
+
+
+@pytest.mark.parametrize("w", ROUTE_CASES, ids=lambda w: f"{w.name}-T{w.T}-D{w.D}-E{w.E}-K{w.K}")
+def test_route(w):
+    wr, bias = wl.router(w, "cpu")
+    x, redrawn = hz.screened_activations(w, wr, bias)
+    assert redrawn <= max(4, 0.05 * w.T)
+    ref_idx, ref_w, ref_logits = oracle.route(hz.bits(x), hz.bits(wr), bias.numpy(), w.K, w.gate_mode)
+    ctx = binding.Context(binding.Shape(w.T, w.D, 64, w.E, w.K, w.S, w.gate_mode, 1))
+    xd, wrd, bd = x.to(DEV), wr.to(DEV), bias.to(DEV)
+    idx = poison_i32(w.T, w.K)
+    wt = torch.full((w.T, w.K), float("nan"), dtype=torch.float32, device=DEV)
+    logits = torch.full((w.T, w.E), float("nan"), dtype=torch.float32, device=DEV)
+    ctx.route_logits(xd, wrd, bd, logits)
+    ctx.route(xd, wrd, bd, idx, wt)
+    ctx.check_status()
+    # the fp32 logits must sit well inside the margin the inputs were screened for
+    assert np.abs(logits.cpu().numpy().astype(np.float64) - ref_logits).max() < hz.TAU / 4
+    assert np.array_equal(idx.cpu().numpy(), ref_idx)
+    got_w = wt.cpu().numpy().astype(np.float64)
+    hz.assert_close_rel_max(got_w, ref_w, "topk_w")
+    assert np.abs(got_w - ref_w).max() < 2e-5
+    assert np.abs(got_w.sum(axis=1) - 1).max() < 1e-5
+
+
+def test_route_no_bias_and_exact_ties():
+    w = small("tiny", T=96, D=128, E=8, K=3, S=8)
+    wr, _ = wl.router(w, "cpu")
+    wr[6] = wr[2]
+    wr[7] = wr[0]
+    x = wl.activations(w, "cpu")
+    logits = oracle.route_logits(hz.bits(x), hz.bits(wr), None)
+    # keep tokens whose only near-ties are the planted exact ones
+    srt = -np.sort(-logits, axis=1)
+    gaps = srt[:, :w.K] - srt[:, 1:w.K + 1]
+    ok = ((gaps == 0) | (gaps >= hz.TAU)).all(axis=1)
+    x = x[torch.from_numpy(np.nonzero(ok)[0])].contiguous()
+    w = w.scaled(T=x.shape[0])
+    ref_idx, ref_w, _ = oracle.route(hz.bits(x), hz.bits(wr), None, w.K, 0)
+    ctx = binding.Context(binding.Shape(w.T, w.D, 64, w.E, w.K, w.S, 0, 1))
+    idx, wt = poison_i32(w.T, w.K), torch.empty(w.T, w.K, dtype=torch.float32, device=DEV)
+    ctx.route(x.to(DEV), wr.to(DEV), None, idx, wt)
+    ctx.check_status()
+    assert np.array_equal(idx.cpu().numpy(), ref_idx)
+    assert any(6 in r or 7 in r for r in ref_idx.tolist())
+
+
+@pytest.mark.parametrize("T,K,E", [(256, 2, 8), (1000, 6, 64), (4096, 8, 256), (1, 1, 1), (77, 3, 3), (0, 2, 8)])
+def test_histogram(T, K, E):
+    rng = np.random.default_rng(T * 31 + E)
+    p = 1.0 / np.arange(1, E + 1) ** 1.2
+    idx = rng.choice(E, size=(T, K), p=p / p.sum()).astype(np.int32)
+    ctx = binding.Context(binding.Shape(T, 64, 64, E, K, max(E, 1), 0, 1))
+    hist = poison_i32(E)
+    ctx.histogram(i32(idx).reshape(T, K), hist)
+    ctx.check_status()
+    assert np.array_equal(hist.cpu().numpy(), oracle.histogram(idx, E))
+    assert int(hist.sum()) == T * K
+
+
+def test_histogram_reports_bad_index_without_faulting():
+    T, K, E = 64, 2, 8
+    idx = np.zeros((T, K), dtype=np.int32)
+    idx[5, 1] = E          # out of range
+    idx[9, 0] = -3
+    ctx = binding.Context(binding.Shape(T, 64, 64, E, K, E, 0, 1))
+    hist = poison_i32(E)
+    ctx.histogram(i32(idx), hist)
+    assert ctx.status() == binding.ERR_BAD_INDEX
+    assert ctx.status() == 0                       # cleared by the read
+    assert int(hist.sum()) == T * K - 2
+
+
+PLAN_CASES = [
+    ([4, 2], 3, 0), ([2, 2], 3, 0), ([4, 2], 4, 0), ([0, 0, 0], 8, 0), ([5, 0, 1], 5, 0), ([3, 3, 3], 3, 0),
+    ([100, 1, 1], 8, 3), ([100, 1], 8, 2), ([9000, 1000, 1000, 1000], 12, 0),
+    ([2 ** 31 - 1, 2 ** 31 - 2, 5], 64, 0),
+]
+
+
+@pytest.mark.parametrize("pred,S,c_max", PLAN_CASES)
+def test_plan_hand_cases(pred, S, c_max):
+    run_plan(np.array(pred, dtype=np.int64), S, c_max)
+
+
+@pytest.mark.parametrize("E,S,seed", [(8, 16, 0), (64, 80, 1), (256, 288, 2), (256, 1024, 3), (1, 9, 4),
+                                      (200, 200, 5), (31, 97, 6)])
+def test_plan_random(E, S, seed):
+    rng = np.random.default_rng(seed)
+    for kind in ("zipf", "ties", "sparse"):
+        if kind == "zipf":
+            pred = np.round(50000 / np.arange(1, E + 1) ** 1.1).astype(np.int64)
+            rng.shuffle(pred)
+        elif kind == "ties":
+            pred = rng.integers(0, 4, size=E) * 12
+        else:
+            pred = np.where(rng.random(E) < 0.7, 0, rng.integers(0, 1000, size=E))
+        run_plan(pred, S, 0)
+        run_plan(pred, S, 3)
+
+
+def run_plan(pred, S, c_max):
+    E = len(pred)
+    ctx = binding.Context(binding.Shape(8, 64, 64, E, 1, S, 0, 1, c_max))
+    rep, so, se, bound = poison_i32(E), poison_i32(E + 1), poison_i32(S), poison_i32(1)
+    ctx.plan(i32(pred), S, rep, so, se, bound)
+    ctx.check_status()
+    r_ref, so_ref, se_ref, b_ref = oracle.plan(pred, S, c_max)
+    assert np.array_equal(rep.cpu().numpy(), r_ref)
+    assert np.array_equal(so.cpu().numpy(), so_ref)
+    assert np.array_equal(se.cpu().numpy(), se_ref)
+    assert int(bound.item()) == b_ref
+
+
+def test_plan_rejects_wrong_slot_count():
+    ctx = binding.Context(binding.Shape(8, 64, 64, 4, 1, 6, 0, 1))
+    n0 = ctx.launch_count()
+    with pytest.raises(binding.MoegpsError) as ei:
+        ctx.plan(i32([1, 2, 3, 4]), 5, poison_i32(4), poison_i32(5), poison_i32(6), poison_i32(1))
+    assert ei.value.code == binding.ERR_INVALID_ARG
+    assert ctx.launch_count() == n0                # nothing was launched
+
+
+DISPATCH_CASES = [
+    # T, D, E, K, S, A, skew
+    (256, 512, 8, 2, 8, 128, 1.0), (256, 512, 8, 2, 8, 1, 1.0), (1000, 256, 8, 2, 16, 128, 1.5),
+    (777, 64, 64, 6, 80, 128, 1.2), (515, 128, 256, 8, 288, 128, 1.0), (515, 128, 256, 8, 288, 1, 1.0),
+    (33, 64, 4, 4, 16, 4, 0.5), (1, 8, 1, 1, 1, 1, 0.0), (300, 72, 5, 1, 9, 32, 2.0), (0, 64, 4, 2, 6, 8, 1.0),
+]
+
+
+@pytest.mark.parametrize("T,D,E,K,S,A,skew", DISPATCH_CASES)
+def test_dispatch(T, D, E, K, S, A, skew):
+    rng = np.random.default_rng(T + 7 * E + S)
+    p = 1.0 / np.arange(1, E + 1) ** skew
+    p /= p.sum()
+    idx = (np.stack([rng.choice(E, size=K, replace=False, p=p) for _ in range(T)]).astype(np.int32)
+           if T else np.zeros((0, K), dtype=np.int32))
+    hist = oracle.histogram(idx, E)
+    pred = np.maximum(0, np.round(hist * (1 + 0.1 * rng.normal(size=E)))).astype(np.int64)
+    rep, so, se, _ = oracle.plan(pred, S)
+    x = rng.integers(0, 1 << 16, size=(T, D), dtype=np.uint16)
+    x[(x & 0x7F80) == 0x7F80] = 0x3F80            # keep the payload finite (bits are the contract)
+    sro_ref, rp_ref, pr_ref, xp_ref = oracle.dispatch(x, idx, hist, rep, so, S, A)
+    shape = binding.Shape(T, D, 64, E, K, S, 0, A)
+    ctx = binding.Context(shape)
+    sro, rp, pr = poison_i32(S + 1), poison_i32(shape.Rcap), poison_i32(T, K)
+    xp = torch.full((shape.Rcap, D), 0x5A5A, dtype=torch.int16, device=DEV).view(torch.bfloat16)
+    ws = torch.full((binding.workspace_bytes(shape),), 0xFF, dtype=torch.uint8, device=DEV)
+    ctx.dispatch(hz.from_bits(x, DEV).reshape(T, D), i32(idx).reshape(T, K), i32(hist), i32(rep), i32(so), sro, rp,
+                 pr, xp, ws)
+    ctx.check_status()
+    assert np.array_equal(sro.cpu().numpy(), sro_ref)
+    assert np.array_equal(rp.cpu().numpy(), rp_ref)
+    assert np.array_equal(pr.cpu().numpy(), pr_ref)
+    got_xp = hz.bits(xp)
+    occ = rp_ref >= 0
+    assert np.array_equal(got_xp[occ], xp_ref[occ])
+    assert (got_xp[~occ] == 0x5A5A).all()          # padding rows are not written
+
+
+def test_dispatch_detects_hist_mismatch():
+    T, D, E, K, S = 64, 64, 4, 2, 6
+    rng = np.random.default_rng(3)
+    idx = np.stack([rng.choice(E, size=K, replace=False) for _ in range(T)]).astype(np.int32)
+    hist = oracle.histogram(idx, E)
+    hist[0] += 1
+    hist[1] -= 1
+    shape = binding.Shape(T, D, 64, E, K, S, 0, 8)
+    ctx = binding.Context(shape)
+    ws = torch.zeros(binding.workspace_bytes(shape), dtype=torch.uint8, device=DEV)
+    ctx.dispatch(torch.zeros(T, D, dtype=torch.bfloat16, device=DEV), i32(idx), i32(hist), i32([2, 2, 1, 1]),
+                 i32([0, 2, 4, 5, 6]), poison_i32(S + 1), poison_i32(shape.Rcap), poison_i32(T, K),
+                 torch.zeros(shape.Rcap, D, dtype=torch.bfloat16, device=DEV), ws)
+    assert ctx.status() == binding.ERR_HIST_MISMATCH
+
+
+def test_dispatch_rejects_small_workspace():
+    shape = binding.Shape(1024, 64, 64, 8, 2, 8, 0, 1)
+    ctx = binding.Context(shape)
+    with pytest.raises(binding.MoegpsError) as ei:
+        ctx.dispatch(None, None, None, None, None, None, None, None, None,
+                     torch.zeros(8, dtype=torch.uint8, device=DEV))
+    assert ei.value.code == binding.ERR_WORKSPACE_TOO_SMALL
+
+
+FFN_CASES = [
+    # T, D, F, E, K, S, A, skew
+    (256, 512, 1024, 8, 2, 8, 128, 1.0),
+    (256, 512, 1024, 8, 2, 12, 1, 1.0),        # unaligned slots: tiles straddle slot ends
+    (300, 256, 384, 4, 2, 7, 128, 1.5),        # F = 3 x 128; D = one 256 tile
+    (200, 320, 200, 6, 3, 9, 128, 1.0),        # D, F not multiples of the tile (ragged K and N tails)
+    (700, 128, 1408, 16, 4, 20, 128, 1.2),     # several row tiles per slot, F = 11 x 128
+    (64, 64, 64, 32, 8, 40, 128, 1.0),         # many almost-empty slots
+    (5, 2048, 256, 2, 1, 2, 128, 0.0),         # long K loop, a handful of rows
+]
+
+
+@pytest.mark.parametrize("T,D,F,E,K,S,A,skew", FFN_CASES)
+def test_expert_ffn(T, D, F, E, K, S, A, skew):
+    rng = np.random.default_rng(T + D + F)
+    p = 1.0 / np.arange(1, E + 1) ** skew
+    p /= p.sum()
+    idx = np.stack([rng.choice(E, size=K, replace=False, p=p) for _ in range(T)]).astype(np.int32)
+    hist = oracle.histogram(idx, E)
+    rep, so, se, _ = oracle.plan(hist, S)
+    x = hz.bits(hz.f64_to_bf16_tensor(rng.normal(size=(T, D))))
+    sro, rp, pr, xp = oracle.dispatch(x, idx, hist, rep, so, S, A)
+    w1 = hz.f64_to_bf16_tensor(rng.normal(size=(E, F, D)) / math.sqrt(D))
+    w3 = hz.f64_to_bf16_tensor(rng.normal(size=(E, F, D)) / math.sqrt(D))
+    w2 = hz.f64_to_bf16_tensor(rng.normal(size=(E, D, F)) / math.sqrt(F))
+    ref = oracle.expert_ffn(xp, sro, se, hz.bits(w1), hz.bits(w3), hz.bits(w2))
+    shape = binding.Shape(T, D, F, E, K, S, 0, A)
+    ctx = binding.Context(shape)
+    # padding rows hold NaN on purpose: rows are independent, so they must not leak into real rows
+    xpd = hz.from_bits(xp, DEV)
+    xpd[torch.from_numpy(rp < 0).to(DEV)] = float("nan")
+    h_ws, yp = poison_bf16(shape.Rcap, F), poison_bf16(shape.Rcap, D)
+    ctx.expert_ffn(xpd, i32(sro), i32(se), w1.to(DEV), w3.to(DEV), w2.to(DEV), h_ws, yp)
+    ctx.check_status()
+    occ = rp >= 0
+    got = yp.float().cpu().numpy().astype(np.float64)
+    hz.assert_close_rel_max(got[occ], ref[occ], "yp")
+    # rows outside every slot's extent stay untouched
+    outside = np.ones(shape.Rcap, dtype=bool)
+    for s in range(S):
+        outside[sro[s]:sro[s + 1]] = False
+    assert torch.isnan(yp[torch.from_numpy(outside).to(DEV)]).all()
+    # bitwise run-to-run determinism
+    yp2 = poison_bf16(shape.Rcap, D)
+    ctx.expert_ffn(xpd, i32(sro), i32(se), w1.to(DEV), w3.to(DEV), w2.to(DEV), h_ws, yp2)
+    ctx.check_status()
+    assert np.array_equal(hz.bits(yp)[occ], hz.bits(yp2)[occ])
+
+
+def test_expert_ffn_zero_gate_weights_give_zero():
+    T, D, F, E = 128, 128, 256, 2
+    shape = binding.Shape(T, D, F, E, 1, E, 0, 128)
+    ctx = binding.Context(shape)
+    g = torch.Generator().manual_seed(1)
+    xp = torch.randn(shape.Rcap, D, generator=g).to(torch.bfloat16).to(DEV)
+    w3 = torch.randn(E, F, D, generator=g).to(torch.bfloat16).to(DEV)
+    w2 = torch.randn(E, D, F, generator=g).to(torch.bfloat16).to(DEV)
+    w1 = torch.zeros(E, F, D, dtype=torch.bfloat16, device=DEV)
+    yp = poison_bf16(shape.Rcap, D)
+    ctx.expert_ffn(xp, i32([0, 128, 256]), i32([1, 0]), w1, w3, w2, poison_bf16(shape.Rcap, F), yp)
+    ctx.check_status()
+    assert (yp[:256] == 0).all()
+
+
+@pytest.mark.parametrize("T,D,K,S,A", [(256, 512, 2, 8, 128), (100, 4096, 2, 8, 1), (77, 2048, 6, 80, 128),
+                                       (33, 7168, 8, 40, 128), (9, 72, 1, 3, 4), (50, 264, 3, 5, 1), (40, 8, 5, 8, 2)])
+def test_combine(T, D, K, S, A):
+    rng = np.random.default_rng(T * D + K)
+    E = S
+    idx = np.stack([rng.choice(E, size=K, replace=False) for _ in range(T)]).astype(np.int32)
+    hist = oracle.histogram(idx, E)
+    rep, so, se, _ = oracle.plan(hist, S)
+    sro, rp, pr, _ = oracle.dispatch(None, idx, hist, rep, so, S, A)
+    shape = binding.Shape(T, D, 64, E, K, S, 0, A)
+    yp = hz.f64_to_bf16_tensor(rng.normal(size=(shape.Rcap, D)))
+    wts = rng.random(size=(T, K)).astype(np.float32)
+    wts /= wts.sum(axis=1, keepdims=True)
+    ref = oracle.combine(hz.bits(yp), pr, wts)
+    ctx = binding.Context(shape)
+    out = poison_bf16(T, D)
+    ctx.combine(yp.to(DEV), i32(pr), torch.from_numpy(wts).to(DEV), out)
+    ctx.check_status()
+    got = out.float().cpu().numpy().astype(np.float64)
+    hz.assert_close_rel_max(got, ref, "out")
+    # fp32 accumulation + one bf16 rounding: within half a bf16 ulp of the reference, plus slack
+    assert np.abs(got - ref).max() <= 2 ** -8 * np.abs(ref).max()
+
+
+def test_invalid_pointers_launch_nothing():
+    shape = binding.Shape(64, 64, 64, 4, 2, 4, 0, 1)
+    ctx = binding.Context(shape)
+    n0 = ctx.launch_count()
+    lib = binding._lib()
+    buf = torch.zeros(4096, dtype=torch.uint8, device=DEV)
+    misaligned = buf.data_ptr() + 4
+    assert lib.moegps_histogram(ctx._h, None, buf.data_ptr(), None) == binding.ERR_INVALID_ARG
+    assert lib.moegps_histogram(ctx._h, misaligned, buf.data_ptr(), None) == binding.ERR_INVALID_ARG
+    assert lib.moegps_combine(ctx._h, buf.data_ptr(), None, buf.data_ptr(), buf.data_ptr(), None) == binding.ERR_INVALID_ARG
+    assert ctx.launch_count() == n0
+    with pytest.raises(TypeError):
+        ctx.histogram(torch.zeros(64, 2, dtype=torch.int64, device=DEV), torch.zeros(4, dtype=torch.int32, device=DEV))
