@@ -54,7 +54,8 @@ typedef enum moegps_error {
   MOEGPS_ERR_UNIMPLEMENTED = -5,
   MOEGPS_ERR_BAD_INDEX = -6,           /* device: an expert/row index outside its range was skipped  */
   MOEGPS_ERR_TIMEOUT = -7,             /* device: a bounded wait inside a kernel ran out             */
-  MOEGPS_ERR_HIST_MISMATCH = -8        /* device: `hist` passed to dispatch disagrees with topk_idx  */
+  MOEGPS_ERR_HIST_MISMATCH = -8,       /* device: `hist` passed to dispatch disagrees with topk_idx  */
+  MOEGPS_ERR_STATIC_SCRATCH_EXCEEDED = -9  /* problem too large for moegps_dispatch_static's built-in scratch */
 } moegps_error;
 
 /* Problem shape, fixed for the life of a context.
@@ -125,6 +126,34 @@ MOEGPS_API int moegps_dispatch(moegps_ctx_t* ctx, const void* x, const int32_t* 
                     const int32_t* replicas, const int32_t* slot_off,
                     int32_t* slot_row_off, int32_t* row_pair, int32_t* pair_row,
                     void* xp, void* workspace, void* stream);
+
+/* dispatch_static - moegps_dispatch without the `workspace` argument.  (The paper has no
+ * counterpart: this is a deployment convenience, not a step of the method.)
+ *
+ * Who needs it: code that must run the shuffle but cannot obtain device memory at that point -
+ * for example a plug-in called inside someone else's serving loop whose memory pool is closed to
+ * it, a caller whose device memory is fully pre-partitioned at start-up, or a real-time path in
+ * which an allocator call (which may block or synchronise the device) is not acceptable.  For them
+ * the scratch that moegps_dispatch takes from the caller is a fixed 1 MiB device array built into
+ * the library (262144 int32 counters).  Every GPU that loads the library holds that 1 MiB until the
+ * process exits, used or not.
+ *
+ * Same inputs, outputs, ordering and error reporting as moegps_dispatch, and bit-identical results.
+ * Differences:
+ *  - Limit: ceil(T*K / 256) * E must not exceed 262144 (the five reference workloads need at most
+ *    32768); beyond it the call returns MOEGPS_ERR_STATIC_SCRATCH_EXCEEDED and launches nothing.
+ *  - The context's device must be the current device of the calling thread (else INVALID_ARG).
+ *  - The first call on each device looks up the array's device address (a host-side query, no
+ *    allocation); make that first call before any stream capture begins.
+ *  - No allocation of any kind is made, here or in the kernels.
+ *  - All calls on a device share the one array, and it keeps whatever the previous call left in
+ *    it.  Nothing in it needs to start at zero (every counter is written before it is read), but
+ *    two calls that may overlap on the GPU (different streams, or different contexts on the same
+ *    device) race on it and corrupt each other: serialise them on one stream or with events. */
+MOEGPS_API int moegps_dispatch_static(moegps_ctx_t* ctx, const void* x, const int32_t* topk_idx,
+                                      const int32_t* hist, const int32_t* replicas, const int32_t* slot_off,
+                                      int32_t* slot_row_off, int32_t* row_pair, int32_t* pair_row,
+                                      void* xp, void* stream);
 
 /* expert_ffn - the expert-parallel SwiGLU FFN (paper, Sections 2 and 3.4) over ragged slots:
  * for every row rho of slot s with e = slot_expert[s]:

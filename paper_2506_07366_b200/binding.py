@@ -49,12 +49,13 @@ class Shape:
 OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA = -1, -2, -3, -4
 ERR_UNIMPLEMENTED, ERR_BAD_INDEX, ERR_TIMEOUT, ERR_HIST_MISMATCH = -5, -6, -7, -8
+ERR_STATIC_SCRATCH_EXCEEDED = -9
 
 EXPORTS = (
     "moegps_create", "moegps_destroy", "moegps_rcap", "moegps_workspace_bytes", "moegps_route",
-    "moegps_route_logits", "moegps_histogram", "moegps_plan", "moegps_dispatch", "moegps_expert_ffn",
-    "moegps_expert_ffn_gate_up", "moegps_expert_ffn_down", "moegps_combine", "moegps_status", "moegps_launch_count", "moegps_last_cuda_error",
-    "moegps_error_string",
+    "moegps_route_logits", "moegps_histogram", "moegps_plan", "moegps_dispatch", "moegps_dispatch_static",
+    "moegps_expert_ffn", "moegps_expert_ffn_gate_up", "moegps_expert_ffn_down", "moegps_combine",
+    "moegps_status", "moegps_launch_count", "moegps_last_cuda_error", "moegps_error_string",
 )
 
 
@@ -95,6 +96,7 @@ def _lib():
         "moegps_histogram": (ctypes.c_int, [vp] * 4),
         "moegps_plan": (ctypes.c_int, [vp, vp, i32, vp, vp, vp, vp, vp]),
         "moegps_dispatch": (ctypes.c_int, [vp] * 12),
+        "moegps_dispatch_static": (ctypes.c_int, [vp] * 11),
         "moegps_expert_ffn": (ctypes.c_int, [vp] * 10),
         "moegps_expert_ffn_gate_up": (ctypes.c_int, [vp] * 8),
         "moegps_expert_ffn_down": (ctypes.c_int, [vp] * 7),
@@ -216,6 +218,24 @@ class Context:
             _ptr(pair_row, torch.int32, (s.T, s.K), "pair_row"),
             _ptr(xp, torch.bfloat16, (s.Rcap, s.D), "xp"),
             _ptr(workspace, workspace.dtype, None, "workspace"), _stream(stream)), "moegps_dispatch")
+
+    def dispatch_static(self, x, topk_idx, hist, replicas, slot_off, slot_row_off, row_pair, pair_row, xp,
+                        stream=None):
+        """dispatch() for callers that cannot hand over a workspace (no allocator available where
+        they run): the scratch is a fixed 1 MiB array inside the library, shared by every call on
+        the device, so overlapping calls must be serialised; ceil(T*K/256)*E must be <= 262144.
+        This method allocates nothing either."""
+        s = self.shape
+        self._check(_lib().moegps_dispatch_static(
+            self._h, _ptr(x, torch.bfloat16, (s.T, s.D), "x"),
+            _ptr(topk_idx, torch.int32, (s.T, s.K), "topk_idx"),
+            _ptr(hist, torch.int32, (s.E,), "hist"),
+            _ptr(replicas, torch.int32, (s.E,), "replicas"),
+            _ptr(slot_off, torch.int32, (s.E + 1,), "slot_off"),
+            _ptr(slot_row_off, torch.int32, (s.S + 1,), "slot_row_off"),
+            _ptr(row_pair, torch.int32, (s.Rcap,), "row_pair"),
+            _ptr(pair_row, torch.int32, (s.T, s.K), "pair_row"),
+            _ptr(xp, torch.bfloat16, (s.Rcap, s.D), "xp"), _stream(stream)), "moegps_dispatch_static")
 
     def expert_ffn(self, xp, slot_row_off, slot_expert, w_gate, w_up, w_down, h_ws, yp, stream=None):
         s = self.shape

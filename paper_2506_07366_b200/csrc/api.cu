@@ -189,6 +189,9 @@ const char* moegps_error_string(int code) {
     case MOEGPS_ERR_BAD_INDEX: return "device saw an index out of range (access skipped)";
     case MOEGPS_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
     case MOEGPS_ERR_HIST_MISMATCH: return "hist passed to dispatch disagrees with topk_idx";
+    case MOEGPS_ERR_STATIC_SCRATCH_EXCEEDED:
+      return "problem too large for the built-in scratch of moegps_dispatch_static (ceil(T*K/256)*E > 262144): "
+             "use moegps_dispatch with a caller-provided workspace";
     default: return "unknown moegps error";
   }
 }

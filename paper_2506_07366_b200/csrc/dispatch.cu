@@ -225,3 +225,53 @@ int moegps_launch_dispatch(moegps_ctx* ctx, const void* x, const int32_t* topk_i
   MOEGPS_AFTER_LAUNCH(ctx);
   return MOEGPS_OK;
 }
+
+// ------------------------------------------------------------------------------------------------
+// moegps_dispatch_static: dispatch for callers that have no allocator to draw the scratch from.
+//
+// The per-segment counters live in the fixed device array below instead of a caller-provided
+// workspace.  The array is part of the library image: every GPU that loads the library holds its
+// 1 MiB until the process exits, whether or not this entry point is ever called.
+namespace {
+
+constexpr size_t kStaticScratchInts = 262144;                    // 1 MiB of int32 counters
+static __device__ __align__(256) int32_t g_dispatch_scratch[kStaticScratchInts];
+
+constexpr int kMaxDevices = 64;
+int32_t* g_scratch_addr[kMaxDevices] = {};                       // device address of the array, per device
+
+}  // namespace
+
+extern "C" MOEGPS_API int moegps_dispatch_static(moegps_ctx_t* ctx, const void* x, const int32_t* topk_idx,
+                                                 const int32_t* hist, const int32_t* replicas,
+                                                 const int32_t* slot_off, int32_t* slot_row_off,
+                                                 int32_t* row_pair, int32_t* pair_row, void* xp, void* stream) {
+  if (!ctx) return MOEGPS_ERR_INVALID_ARG;
+  const moegps_shape_t& s = ctx->shape;
+  const void* always[] = {hist, replicas, slot_off, slot_row_off};
+  for (const void* p : always)
+    if (!p || !moegps_aligned16(p)) return MOEGPS_ERR_INVALID_ARG;
+  if (s.T > 0) {
+    const void* with_tokens[] = {x, topk_idx, pair_row, xp};
+    for (const void* p : with_tokens)
+      if (!p || !moegps_aligned16(p)) return MOEGPS_ERR_INVALID_ARG;
+  }
+  if (moegps_rcap_of(s) > 0 && (!row_pair || !moegps_aligned16(row_pair))) return MOEGPS_ERR_INVALID_ARG;
+  // the scratch holds one int32 per (segment, expert); larger problems must use moegps_dispatch
+  const int64_t R = (int64_t)s.T * s.K;
+  const int64_t nseg = (R + kSegPairs - 1) / kSegPairs;
+  if ((uint64_t)(nseg * s.E) > kStaticScratchInts) return MOEGPS_ERR_STATIC_SCRATCH_EXCEEDED;
+  int dev = -1;
+  MOEGPS_CUDA_TRY(ctx, cudaGetDevice(&dev));
+  if (dev != ctx->device || dev < 0 || dev >= kMaxDevices) return MOEGPS_ERR_INVALID_ARG;
+  if (!g_scratch_addr[dev]) {
+    // In host code the array's name is only a handle; the address a kernel can use has to be asked
+    // for, once per device, with that device current.
+    int32_t* p = nullptr;
+    MOEGPS_CUDA_TRY(ctx, cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_dispatch_scratch));
+    if (!p) return MOEGPS_ERR_CUDA;
+    g_scratch_addr[dev] = p;
+  }
+  return moegps_launch_dispatch(ctx, x, topk_idx, hist, replicas, slot_off, slot_row_off, row_pair, pair_row, xp,
+                                g_scratch_addr[dev], (cudaStream_t)stream);
+}
