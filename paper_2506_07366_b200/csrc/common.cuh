@@ -28,6 +28,7 @@ struct moegps_ctx {
   const void* rt_key[2];
   CUtensorMap tm_rx, tm_rw;
   bool rt_valid;
+  bool route_attr_done;
 };
 
 #define MOEGPS_CUDA_TRY(ctx, expr)                                   \

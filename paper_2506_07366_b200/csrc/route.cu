@@ -1,59 +1,203 @@
 // route: router GEMM fused with bias, warp-shuffle top-K and the gate weights (paper, Section 2).
-// One warp per token: the lanes split the model dimension (128-bit loads of X and of the router
-// rows), partial dot products are reduced by shuffles into a per-warp logit row in shared memory,
-// and the warp then selects the K largest logits (route_epilogue.cuh).
+//
+// logits[128 tokens, E] = X_tile * Wr^T on the 5th-generation tensor cores: the token tile is the
+// MMA's M (128 rows), the experts its N (E rounded up to 16, at most 256), accumulators in TMEM.
+// The kernel is bound by reading X once from HBM, so the grid must cover the chip even when
+// T/128 is small: the model dimension is split over the KS CTAs of a thread-block cluster
+// (grid = token tiles x KS).  Each CTA streams its slice of X and Wr through a TMA -> shared-memory
+// ring into tcgen05.mma, parks its fp32 partial logits in its own shared memory, and after a
+// cluster barrier CTA r reduces rows [r*128/KS, (r+1)*128/KS) over all KS partials through
+// distributed shared memory in a fixed order (deterministic), adds the bias and lets one warp per
+// token select the top K by shuffles (route_epilogue.cuh).
+// Warp roles in the main loop: warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
+// warps 2..5 = TMEM -> shared-memory drain.  Every mbarrier wait is bounded.
 #include "common.cuh"
 #include "route_epilogue.cuh"
+#include "sm100.cuh"
+
+bool moegps_make_tmap_2d(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 
 namespace {
 
-constexpr int kWarpsPerBlock = 8;
-constexpr int kThreads = kWarpsPerBlock * 32;
-constexpr int kMaxE = 256;
-constexpr int kEG = 8;     // experts per pass over the token row
+using namespace sm100;
 
-__device__ __forceinline__ void dot8(float& acc, const uint4& a, const uint4& b) {
-  const uint32_t ua[4] = {a.x, a.y, a.z, a.w}, ub[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    acc = fmaf(__uint_as_float(ua[i] << 16), __uint_as_float(ub[i] << 16), acc);
-    acc = fmaf(__uint_as_float(ua[i] & 0xffff0000u), __uint_as_float(ub[i] & 0xffff0000u), acc);
-  }
+constexpr int BM = 128;
+constexpr int BK = 64;
+constexpr int kThreads = 192;
+constexpr int kABytes = BM * BK * 2;      // 16 KiB of X per stage
+constexpr int kMaxE = 256;
+
+struct RouteParams {
+  int T, D, E, K, gate_mode;
+  int e_pad;        // E rounded up to a multiple of 16
+  int stages;
+  int ks;           // cluster size = number of K slices
+  int kb_per_cta;   // 64-wide K blocks per slice
+  int tmem_cols;
+  int ring_bytes;   // stages * (kABytes + e_pad * 128)
+  int part_stride;  // floats per row of the partial-logit buffer (e_pad + 1: conflict-free)
+};
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Address of `local_smem_addr` in the shared memory of CTA `rank` of this cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+  return v;
 }
 
-__global__ void __launch_bounds__(kThreads)
-route_kernel(const uint4* __restrict__ x, const uint4* __restrict__ wr, const float* __restrict__ bias, int T,
-             int chunks /* D/8 */, int E, int K, int gate_mode, int32_t* __restrict__ topk_idx,
-             float* __restrict__ topk_w, float* __restrict__ logits_out) {
-  __shared__ float logit[kWarpsPerBlock][kMaxE];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int t = blockIdx.x * kWarpsPerBlock + warp;
-  if (t >= T) return;
-  const uint4* xr = x + (int64_t)t * chunks;
-  for (int e0 = 0; e0 < E; e0 += kEG) {
-    float acc[kEG];
-#pragma unroll
-    for (int i = 0; i < kEG; ++i) acc[i] = 0.f;
-    for (int c = lane; c < chunks; c += 32) {
-      const uint4 xv = xr[c];
-#pragma unroll
-      for (int i = 0; i < kEG; ++i)
-        if (e0 + i < E) dot8(acc[i], xv, wr[(int64_t)(e0 + i) * chunks + c]);
+__global__ void __launch_bounds__(kThreads, 1)
+route_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
+             const RouteParams p, const float* __restrict__ bias, int32_t* __restrict__ topk_idx,
+             float* __restrict__ topk_w, float* __restrict__ logits_out, int32_t* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  // [ ring (re-used as the partial-logit buffer) | per-warp logit rows | barriers ]
+  const int part_bytes = BM * p.part_stride * 4;
+  const int region0 = p.ring_bytes > part_bytes ? p.ring_bytes : part_bytes;
+  float* partial = reinterpret_cast<float*>(smem);
+  float* warp_logit = reinterpret_cast<float*>(smem + region0);                 // [6][kMaxE]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + region0 + 6 * kMaxE * 4);
+  uint64_t* full = bars;                 // [stages]
+  uint64_t* empty = bars + p.stages;     // [stages]
+  uint64_t* acc_full = bars + 2 * p.stages;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * p.stages + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int m0 = blockIdx.x * BM;
+  const int nkb = (p.D + BK - 1) / BK;
+  const int kb_begin = (int)rank * p.kb_per_cta;
+  const int kb_end = min(nkb, kb_begin + p.kb_per_cta);
+  const int stage_bytes = kABytes + p.e_pad * 128;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < p.stages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+    mbar_init(acc_full, 1);
+    *abort_flag = 0;
+    fence_mbar_init();
+    prefetch_tensormap(&tm_x);
+    prefetch_tensormap(&tm_w);
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, (uint32_t)p.tmem_cols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int kb = kb_begin; kb < kb_end; ++kb) {
+        if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag)) break;
+        uint8_t* sa = smem + (size_t)stage * stage_bytes;
+        mbar_arrive_expect_tx(&full[stage], (uint32_t)stage_bytes);
+        tma_load_2d(sa, &tm_x, &full[stage], kb * BK, m0);
+        tma_load_2d(sa + kABytes, &tm_w, &full[stage], kb * BK, 0);
+        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+      }
     }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = idesc_bf16_f32(BM, p.e_pad);
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int kb = kb_begin; kb < kb_end; ++kb) {
+        if (!mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
+        tc_fence_after_sync();
+        const uint32_t sa = smem_u32(smem + (size_t)stage * stage_bytes);
+        const uint64_t da = smem_desc_k_sw128(sa);
+        const uint64_t db = smem_desc_k_sw128(sa + kABytes);
 #pragma unroll
-    for (int i = 0; i < kEG; ++i) {
-      float v = acc[i];
-#pragma unroll
-      for (int m = 16; m >= 1; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
-      if (lane == 0 && e0 + i < E) logit[warp][e0 + i] = v + (bias ? bias[e0 + i] : 0.f);
+        for (int k = 0; k < BK / 16; ++k)
+          mma_bf16(tmem_base, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb > kb_begin) || k > 0);
+        mma_commit(&empty[stage]);
+        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+      }
+      if (ok && kb_begin < kb_end) mma_commit(acc_full);
     }
+  } else {
+    // drain this CTA's partial logits: thread = token row, 32 columns per TMEM load
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    float* prow0 = partial + (size_t)row * p.part_stride;
+    if (kb_begin >= kb_end) {
+      // an empty K slice (only when D is short): its partial is zero
+      for (int c = 0; c < p.e_pad; ++c) prow0[c] = 0.f;
+    }
+    const bool ok = kb_begin < kb_end && mbar_wait(acc_full, 0, abort_flag);
+    tc_fence_after_sync();
+    if (ok) {
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+      float* prow = partial + (size_t)row * p.part_stride;
+      for (int c0 = 0; c0 < p.e_pad; c0 += 32) {
+        uint32_t v[32];
+        tmem_ld32(taddr + c0, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+          if (c0 + i < p.e_pad) prow[c0 + i] = __uint_as_float(v[i]);
+      }
+    }
+    tc_fence_before_sync();
   }
   __syncwarp();
-  if (logits_out) {
-    for (int e = lane; e < E; e += 32) logits_out[(int64_t)t * E + e] = logit[warp][e];
-    if (!topk_idx) return;
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) {
+    moegps_report(status, MOEGPS_ERR_TIMEOUT, (int)blockIdx.x);
+    for (int i = 0; i < 1000; ++i) __nanosleep(1000);    // let copies still in flight land
   }
-  warp_topk_gate<kMaxE / 32>(logit[warp], E, K, gate_mode, topk_idx + (int64_t)t * K, topk_w + (int64_t)t * K);
+  __syncwarp();
+  cluster_sync_all();           // every CTA's partial is complete and visible cluster-wide
+
+  // reduction + selection: CTA `rank` owns rows [rank*rows_per, (rank+1)*rows_per) of the tile
+  {
+    const int rows_per = BM / p.ks;
+    float* mylogit = warp_logit + warp * kMaxE;
+    const uint32_t part_u32 = smem_u32(partial);
+    for (int r = warp; r < rows_per; r += kThreads / 32) {
+      const int row = (int)rank * rows_per + r;
+      const int t = m0 + row;
+      if (t < p.T) {                                     // warp-uniform
+        for (int e = lane; e < p.E; e += 32) {
+          float acc = 0.f;
+          const uint32_t off = part_u32 + (uint32_t)((row * p.part_stride + e) * 4);
+          for (int k = 0; k < p.ks; ++k) acc += ld_cluster_f32(map_to_cta(off, (uint32_t)k));
+          mylogit[e] = acc + (bias ? bias[e] : 0.f);
+        }
+        __syncwarp();
+        if (logits_out)
+          for (int e = lane; e < p.E; e += 32) logits_out[(int64_t)t * p.E + e] = mylogit[e];
+        if (topk_idx)
+          warp_topk_gate<kMaxE / 32>(mylogit, p.E, p.K, p.gate_mode, topk_idx + (int64_t)t * p.K,
+                                     topk_w + (int64_t)t * p.K);
+        __syncwarp();
+      }
+    }
+  }
+  cluster_sync_all();           // nobody leaves while a peer may still read its shared memory
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+  }
 }
 
 }  // namespace
@@ -61,9 +205,61 @@ route_kernel(const uint4* __restrict__ x, const uint4* __restrict__ wr, const fl
 int moegps_launch_route(moegps_ctx* ctx, const void* x, const void* wr, const float* bias, int32_t* topk_idx,
                         float* topk_w, float* logits_out, cudaStream_t st) {
   const moegps_shape_t& s = ctx->shape;
-  const int blocks = (s.T + kWarpsPerBlock - 1) / kWarpsPerBlock;
-  route_kernel<<<blocks, kThreads, 0, st>>>(static_cast<const uint4*>(x), static_cast<const uint4*>(wr), bias, s.T,
-                                            s.D / 8, s.E, s.K, s.gate_mode, topk_idx, topk_w, logits_out);
-  MOEGPS_AFTER_LAUNCH(ctx);
+  RouteParams p;
+  p.T = s.T; p.D = s.D; p.E = s.E; p.K = s.K; p.gate_mode = s.gate_mode;
+  p.e_pad = (s.E + 15) / 16 * 16;
+  const int stage_bytes = kABytes + p.e_pad * 128;
+  p.stages = 196608 / stage_bytes;          // ring of at most 192 KiB
+  if (p.stages > 8) p.stages = 8;
+  const int nkb = (s.D + BK - 1) / BK;
+  const int tiles = (s.T + BM - 1) / BM;
+  // split the model dimension until the grid covers most of the chip (cluster size <= 8, a power
+  // of two so that 128 rows divide evenly, and every slice keeps at least 4 K blocks)
+  int ks = 1;
+  while (ks < 8 && tiles * ks * 2 <= ctx->sm_count + ctx->sm_count / 4 && nkb / (ks * 2) >= 4) ks *= 2;
+  p.ks = ks;
+  p.kb_per_cta = (nkb + ks - 1) / ks;
+  if (p.stages > p.kb_per_cta) p.stages = p.kb_per_cta < 2 ? 2 : p.kb_per_cta;
+  p.tmem_cols = 32;
+  while (p.tmem_cols < p.e_pad) p.tmem_cols *= 2;
+  p.ring_bytes = p.stages * stage_bytes;
+  p.part_stride = p.e_pad + 1;
+  const int part_bytes = BM * p.part_stride * 4;
+  const int region0 = p.ring_bytes > part_bytes ? p.ring_bytes : part_bytes;
+  const size_t smem_bytes = 1024 + (size_t)region0 + 6 * kMaxE * 4 + (2 * p.stages + 1) * 8 + 64;
+
+  if (!(ctx->rt_valid && ctx->rt_key[0] == x && ctx->rt_key[1] == wr)) {
+    ctx->rt_valid = false;
+    if (!(moegps_make_tmap_2d(&ctx->tm_rx, x, (uint64_t)s.T, (uint64_t)s.D, BM) &&
+          moegps_make_tmap_2d(&ctx->tm_rw, wr, (uint64_t)s.E, (uint64_t)s.D, (uint32_t)p.e_pad))) {
+      ctx->last_cuda_error = (int)cudaErrorInvalidValue;
+      return MOEGPS_ERR_CUDA;
+    }
+    ctx->rt_key[0] = x; ctx->rt_key[1] = wr;
+    ctx->rt_valid = true;
+  }
+  if (!ctx->route_attr_done) {
+    MOEGPS_CUDA_TRY(ctx, cudaFuncSetAttribute(route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    ctx->route_attr_done = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)tiles, (unsigned)ks, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem_bytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 1;
+  attr[0].val.clusterDim.y = (unsigned)ks;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, route_kernel, ctx->tm_rx, ctx->tm_rw, p, bias, topk_idx, topk_w,
+                                     logits_out, ctx->d_status);
+  ctx->launches += 1;
+  if (e != cudaSuccess) {
+    ctx->last_cuda_error = (int)e;
+    return MOEGPS_ERR_CUDA;
+  }
   return MOEGPS_OK;
 }
