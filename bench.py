@@ -30,6 +30,10 @@ from paper_2506_07366_b200 import workloads as wl  # noqa: E402
 METRIC = "moe_layer_tokens_per_s"
 UNIT = "tokens/s"
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one gate+up GEMM launch, from the ncu captures
+# summarised under profiles/ (bytes; None = not captured for the current kernel)
+GATE_UP_DRAM_TRAFFIC = {}
+
 
 # ------------------------------------------------------------------------------------- helpers
 def measured_peaks():
@@ -103,6 +107,27 @@ def visible_gpu_index(local_rank: int) -> int:
     return local_rank
 
 
+# ------------------------------------------------------------------------------------- multi-rank plumbing
+def rank_workload(w, rank: int):
+    """The workload whose activations rank `rank` draws: same shapes and recipe, its own seed, so
+    that every rank processes a different batch (data-parallel replicas, no data-path collective)."""
+    return w.scaled(number=w.number + 50 * rank)
+
+
+def max_over_ranks(ms: float, dist, device) -> float:
+    """The job is as slow as its slowest rank."""
+    if dist is None:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(world: int, tokens_per_rank: int, steps: int, elapsed_ms: float) -> float:
+    """Tokens per second over all ranks (weak scaling: every rank processes tokens_per_rank per step)."""
+    return world * tokens_per_rank * steps / (elapsed_ms * 1e-3)
+
+
 # ------------------------------------------------------------------------------------- our arm
 def run_ours(args):
     from paper_2506_07366_b200 import binding
@@ -128,7 +153,7 @@ def run_ours(args):
     # every rank draws its own batch (same weights: data parallel replicas of the layer)
     wr, bias = wl.router(w, dev)
     w1, w3, w2 = wl.expert_weights(w, dev)
-    x = wl.activations(w.scaled(number=w.number + 50 * rank), dev)
+    x = wl.activations(rank_workload(w, rank), dev)
     layer = MoeLayer(shape, wr, bias, w1, w3, w2, device=local_rank)
     ctx = layer.ctx
 
@@ -196,11 +221,8 @@ def run_ours(args):
     launches = ctx.launch_count() - launches0
     clocks = sampler.stop() if rank == 0 else None
     ctx.check_status()
-    if dist is not None:
-        tmax = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(tmax.item())
-    value = world * w.T * args.steps / (elapsed_ms * 1e-3)
+    elapsed_ms = max_over_ranks(elapsed_ms, dist, dev)
+    value = whole_job_rate(world, w.T, args.steps, elapsed_ms)
 
     gate_up_ms = statistics.mean(a.elapsed_time(b) for a, b, _ in gemm_marks)
     down_ms = statistics.mean(b.elapsed_time(c) for _, b, c in gemm_marks)
@@ -220,12 +242,9 @@ def run_ours(args):
     e1.record(stream)
     barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if dist is not None:
-        tmax = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tmax.item())
+    e2e_ms = max_over_ranks(e2e_ms, dist, dev)
     ctx.check_status()
-    e2e_value = world * w.T * args.steps / (e2e_ms * 1e-3)
+    e2e_value = whole_job_rate(world, w.T, args.steps, e2e_ms)
 
     if rank != 0:
         if dist is not None:
@@ -233,10 +252,17 @@ def run_ours(args):
         return
 
     peaks = measured_peaks()
+    kernels = per_call_timings(ctx, layer, w, x, wr, bias, w1, w3, w2, pred_dev, peaks) if world == 1 else None
     flops_gate_up = 4.0 * w.R * w.D * w.F          # two of the three SwiGLU GEMMs, 2*R*D*F each
     achieved = flops_gate_up / (gate_up_ms * 1e-3) / 1e12
     ffn_tflops = 6.0 * w.R * w.D * w.F / ((gate_up_ms + down_ms) * 1e-3) / 1e12
     hist_np = true_hist.numpy().astype("float64")
+    # a timed region of a few hundred ms runs at boost clocks: the burst peak is the fair denominator;
+    # from a couple of seconds on, the power cap has settled and the sustained peak applies
+    if elapsed_ms >= 2000.0:
+        peak, peak_kind = peaks["bf16_sustained"], " (sustained bf16 GEMM: timed region >= 2 s)"
+    else:
+        peak, peak_kind = peaks["bf16_burst"], " (burst bf16 GEMM: timed region < 2 s, boost clocks)"
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
@@ -251,18 +277,69 @@ def run_ours(args):
         "gpu_launches": int(launches),
         "clocks": clocks,
         "roofline": {"kernel": "grouped_gemm_kernel<SwiGLU> (expert_ffn gate+up)", "bound": "tensor",
-                     "achieved": achieved, "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
-                     "frac": achieved / peaks["bf16_sustained"], "frac_of_burst_peak": achieved / peaks["bf16_burst"],
-                     "peak_source": peaks["source"] + " (sustained bf16, kernel timed inside the step)",
-                     "ms_per_launch": gate_up_ms, "traffic": None},
+                     "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                     "frac_of_burst_peak": achieved / peaks["bf16_burst"],
+                     "frac_of_sustained_peak": achieved / peaks["bf16_sustained"],
+                     "peak_source": peaks["source"] + peak_kind,
+                     "ms_per_launch": gate_up_ms, "traffic": GATE_UP_DRAM_TRAFFIC.get(w.name)},
         "expert_ffn": {"tflops": ffn_tflops, "gate_up_ms": gate_up_ms, "down_ms": down_ms,
                        "frac_of_sustained_peak": ffn_tflops / peaks["bf16_sustained"]},
     }
+    if kernels is not None:
+        line["calls_cold_l2"] = kernels
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(w, x, wr, bias, w1, w3, w2, pred)
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
+
+
+def per_call_timings(ctx, layer, w, x, wr, bias, w1, w3, w2, pred_dev, peaks, iters=7):
+    """Each library call timed alone (CUDA events on the launching stream, median of `iters`) with L2
+    flushed before every call by overwriting a 512 MB buffer, against the call's algorithmic HBM bytes
+    or flops.  These explain the step time; they are not part of the timed step."""
+    stream = torch.cuda.current_stream()
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=x.device)
+    R, T, D, F, E, K = w.R, w.T, w.D, w.F, w.E, w.K
+    ctx.plan(pred_dev, w.S, layer.replicas, layer.slot_off, layer.slot_expert, layer.bound)
+    calls = [
+        ("plan", lambda: ctx.plan(pred_dev, w.S, layer.replicas, layer.slot_off, layer.slot_expert, layer.bound),
+         None, None),
+        ("route", lambda: ctx.route(x, wr, bias, layer.topk_idx, layer.topk_w),
+         2.0 * T * D + 2.0 * E * D + 8.0 * T * K, 2.0 * T * D * E),
+        ("histogram", lambda: ctx.histogram(layer.topk_idx, layer.hist), 4.0 * R, None),
+        ("dispatch", lambda: ctx.dispatch(x, layer.topk_idx, layer.hist, layer.replicas, layer.slot_off,
+                                          layer.slot_row_off, layer.row_pair, layer.pair_row, layer.xp,
+                                          layer.workspace), 2.0 * T * D + 2.0 * R * D + 12.0 * R, None),
+        ("expert_ffn_gate_up", lambda: ctx.expert_ffn_gate_up(layer.xp, layer.slot_row_off, layer.slot_expert, w1, w3,
+                                                              layer.h_ws), None, 4.0 * R * D * F),
+        ("expert_ffn_down", lambda: ctx.expert_ffn_down(layer.h_ws, layer.slot_row_off, layer.slot_expert, w2,
+                                                        layer.yp), None, 2.0 * R * D * F),
+        ("combine", lambda: ctx.combine(layer.yp, layer.pair_row, layer.topk_w, layer.out),
+         2.0 * R * D + 2.0 * T * D + 8.0 * R, None),
+    ]
+    out = {}
+    for name, fn, nbytes, flops in calls:
+        times = []
+        for _ in range(iters):
+            flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            b.synchronize()
+            times.append(a.elapsed_time(b))
+        ms = statistics.median(times)
+        rec = {"us": ms * 1e3}
+        if nbytes is not None:
+            rec["gbs"] = nbytes / (ms * 1e-3) / 1e9
+            rec["frac_of_hbm_peak"] = rec["gbs"] / peaks["hbm_gbs"]
+        if flops is not None and name.startswith("expert"):
+            rec["tflops"] = flops / (ms * 1e-3) / 1e12
+            rec["frac_of_burst_peak"] = rec["tflops"] / peaks["bf16_burst"]
+        out[name] = rec
+    ctx.check_status()
+    return out
 
 
 # ------------------------------------------------------------------------------------- oracle arm

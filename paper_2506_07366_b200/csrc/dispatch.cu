@@ -1,14 +1,16 @@
 // dispatch: the routing shuffle on one device (paper, Section 2; replica choice of Algorithm 1).
 //
-// The flat pair list is cut into segments of kSegPairs consecutive pairs, one warp per segment.
-//   1. segment_count : per-segment, per-expert pair counts -> workspace[seg][e]; row_pair := -1
-//   2. scan_offsets  : per expert an exclusive scan of the counts over segments (in place), and the
-//                      slot row offsets from hist / replicas / row_align (block scan)
-//   3. scatter_index : every warp re-walks its segment in pair order; the stable rank of a pair is
-//                      the segment's base plus the number of earlier same-expert pairs in the segment
-//                      (warp match + running counters), from which replica, slot and row follow
-//   4. copy_rows     : one warp per token reads the token row once (128-bit loads) and writes it to
-//                      its K rows of the permuted buffer (128-bit stores)
+// The flat pair list is cut into segments of kSegPairs consecutive pairs.  Two kernels:
+//   1. count_scan : one CTA per segment counts its pairs per expert (warp match + shared counters)
+//                   into workspace[seg][e] and fills row_pair with -1; the CTA that finishes last
+//                   (ticket counter, no waiting) turns the counts into per-expert exclusive prefix
+//                   sums over the segments and derives the slot row offsets from hist / replicas /
+//                   row_align with a block scan
+//   2. rank_copy  : one warp per token.  The stable rank of a pair is its segment's base plus the
+//                   number of earlier same-expert pairs inside the segment, which the warp counts
+//                   from the segment's indices (a 1 KiB read); replica, slot and row follow in
+//                   integer arithmetic.  The warp then reads the token row once (128-bit loads) and
+//                   writes it to its K rows of the permuted buffer (128-bit stores).
 // Stable by construction, integer only, no atomics on results => bit-exact and deterministic.
 #include "common.cuh"
 
@@ -18,22 +20,29 @@ constexpr int kWarpsPerBlock = 8;
 constexpr int kThreads = kWarpsPerBlock * 32;
 constexpr int kMaxE = 256;
 constexpr int kMaxS = 1024;
+constexpr int kScanThreads = 1024;
 
-__global__ void __launch_bounds__(kThreads)
-segment_count_kernel(const int32_t* __restrict__ topk_idx, int64_t R, int E, int32_t* __restrict__ seg_cnt,
-                     int nseg, int32_t* __restrict__ row_pair, int64_t Rcap, int32_t* __restrict__ status) {
-  __shared__ int32_t cnt[kWarpsPerBlock][kMaxE];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  // padding rows keep -1: fill everything, occupied rows are overwritten by scatter_index
-  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < Rcap; i += (int64_t)gridDim.x * blockDim.x)
+static_assert(kSegPairs == 256, "count_scan assigns one of its first 256 threads to each pair of a segment");
+
+__global__ void __launch_bounds__(kScanThreads)
+count_scan_kernel(const int32_t* __restrict__ topk_idx, int64_t R, int E, int S, int A,
+                  int32_t* seg_cnt, int nseg, int32_t* __restrict__ row_pair, int64_t Rcap,
+                  const int32_t* __restrict__ hist, const int32_t* __restrict__ replicas,
+                  const int32_t* __restrict__ slot_off, int32_t* __restrict__ slot_row_off,
+                  int32_t* status) {
+  __shared__ int32_t cnt[kMaxE];
+  __shared__ int32_t padded[kMaxS];     // rows reserved for each slot (load rounded up to A)
+  __shared__ int32_t warp_tot[32];
+  __shared__ int is_last;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int seg = blockIdx.x;
+  // padding rows keep -1: fill everything, occupied rows are overwritten by rank_copy
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + tid; i < Rcap; i += (int64_t)gridDim.x * blockDim.x)
     row_pair[i] = -1;
-  const int seg = blockIdx.x * kWarpsPerBlock + warp;
-  if (seg >= nseg) return;
-  for (int e = lane; e < E; e += 32) cnt[warp][e] = 0;
-  __syncwarp();
-  const int64_t p0 = (int64_t)seg * kSegPairs;
-  for (int it = 0; it < kSegPairs / 32; ++it) {
-    const int64_t p = p0 + it * 32 + lane;
+  if (tid < E) cnt[tid] = 0;
+  __syncthreads();
+  if (tid < kSegPairs) {                      // warps 0..7, whole warps
+    const int64_t p = (int64_t)seg * kSegPairs + tid;
     int e = -1;
     if (p < R) {
       e = topk_idx[p];
@@ -43,29 +52,30 @@ segment_count_kernel(const int32_t* __restrict__ topk_idx, int64_t R, int E, int
       }
     }
     const unsigned same = __match_any_sync(0xffffffffu, e);
-    if (e >= 0 && lane == (31 - __clz(same))) cnt[warp][e] += __popc(same);   // one leader per expert
-    __syncwarp();
+    if (e >= 0 && lane == (31 - __clz(same))) atomicAdd(&cnt[e], __popc(same));   // one add per warp and expert
   }
-  for (int e = lane; e < E; e += 32) seg_cnt[(int64_t)seg * E + e] = cnt[warp][e];
-}
+  __syncthreads();
+  if (tid < E && seg < nseg) seg_cnt[(int64_t)seg * E + tid] = cnt[tid];
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const int ticket = atomicAdd(&status[2], 1);
+    is_last = ticket == (int)gridDim.x - 1;
+    if (is_last) status[2] = 0;               // ready for the next call
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
 
-// One CTA of 1024 threads.
-__global__ void __launch_bounds__(1024)
-scan_offsets_kernel(int32_t* __restrict__ seg_cnt, int nseg, int E, int S, int A,
-                    const int32_t* __restrict__ hist, const int32_t* __restrict__ replicas,
-                    const int32_t* __restrict__ slot_off, int32_t* __restrict__ slot_row_off,
-                    int32_t* __restrict__ status) {
-  __shared__ int32_t padded[kMaxS];     // rows reserved for each slot (load rounded up to A)
-  __shared__ int32_t warp_tot[32];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // ---- last CTA only: every segment's counts are now visible ----
   for (int s = tid; s < S; s += blockDim.x) padded[s] = 0;
   __syncthreads();
   // (a) per expert: exclusive scan of its counts over the segments; lanes stride the segments
-  for (int e = warp; e < E; e += 32) {
+  for (int e = warp; e < E; e += kScanThreads / 32) {
     int running = 0;
     for (int g0 = 0; g0 < nseg; g0 += 32) {
       const int g = g0 + lane;
-      const int c = g < nseg ? seg_cnt[(int64_t)g * E + e] : 0;
+      const int c = g < nseg ? __ldcg(&seg_cnt[(int64_t)g * E + e]) : 0;
       int incl = c;
 #pragma unroll
       for (int d = 1; d < 32; d <<= 1) {
@@ -109,92 +119,86 @@ scan_offsets_kernel(int32_t* __restrict__ seg_cnt, int nseg, int E, int S, int A
 }
 
 __global__ void __launch_bounds__(kThreads)
-scatter_index_kernel(const int32_t* __restrict__ topk_idx, int64_t R, int E, int S, int64_t Rcap,
-                     const int32_t* __restrict__ seg_base, int nseg, const int32_t* __restrict__ hist,
-                     const int32_t* __restrict__ replicas, const int32_t* __restrict__ slot_off,
-                     const int32_t* __restrict__ slot_row_off, int32_t* __restrict__ pair_row,
-                     int32_t* __restrict__ row_pair, int32_t* __restrict__ status) {
-  __shared__ int32_t running[kWarpsPerBlock][kMaxE];
-  __shared__ int32_t s_hist[kMaxE], s_rep[kMaxE], s_so[kMaxE];
-  __shared__ int32_t s_sro[kMaxS + 1];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (int e = threadIdx.x; e < E; e += blockDim.x) {
-    s_hist[e] = hist[e];
-    s_rep[e] = replicas[e];
-    s_so[e] = slot_off[e];
-  }
-  for (int s = threadIdx.x; s <= S; s += blockDim.x) s_sro[s] = slot_row_off[s];
-  const int seg = blockIdx.x * kWarpsPerBlock + warp;
-  if (seg < nseg)
-    for (int e = lane; e < E; e += 32) running[warp][e] = seg_base[(int64_t)seg * E + e];
-  __syncthreads();
-  if (seg >= nseg) return;
-  const int64_t p0 = (int64_t)seg * kSegPairs;
-  const unsigned lt = (1u << lane) - 1u;
-  for (int it = 0; it < kSegPairs / 32; ++it) {
-    const int64_t p = p0 + it * 32 + lane;
-    int e = -1;
-    if (p < R) {
-      e = topk_idx[p];
-      if (e < 0 || e >= E) e = -1;       // already reported by segment_count
-    }
-    const unsigned same = __match_any_sync(0xffffffffu, e);
-    int rank = 0;
-    if (e >= 0) rank = running[warp][e] + __popc(same & lt);
-    __syncwarp();
-    if (e >= 0 && lane == (31 - __clz(same))) running[warp][e] += __popc(same);
-    __syncwarp();
-    if (e >= 0) {
-      const long long n = s_hist[e];
-      const int r = s_rep[e];
-      if (n <= 0 || r < 1 || rank >= n) {
-        moegps_report(status, MOEGPS_ERR_HIST_MISMATCH, e);
-      } else {
-        const int rho = (int)((((long long)rank + 1) * r - 1) / n);   // replica whose range holds `rank`
-        const int start = (int)(((long long)rho * n) / r);
-        const int slot = s_so[e] + rho;
-        const long long row = slot <= S - 1 && slot >= 0 ? (long long)s_sro[slot] + (rank - start) : -1;
-        if (row < 0 || row >= Rcap) {
-          moegps_report(status, MOEGPS_ERR_BAD_INDEX, (int)(p & 0x7fffffff));
-        } else {
-          pair_row[p] = (int32_t)row;
-          row_pair[row] = (int32_t)p;
-        }
-      }
-    }
-  }
-}
-
-__global__ void __launch_bounds__(kThreads)
-copy_rows_kernel(const uint4* __restrict__ x, int T, int K, int chunks /* D*2/16 */,
-                 const int32_t* __restrict__ pair_row, int64_t Rcap, uint4* __restrict__ xp) {
+rank_copy_kernel(const uint4* __restrict__ x, int T, int K, int chunks /* D*2/16 */,
+                 const int32_t* __restrict__ topk_idx, int64_t R, int E, int S, int64_t Rcap,
+                 const int32_t* __restrict__ seg_base, const int32_t* __restrict__ hist,
+                 const int32_t* __restrict__ replicas, const int32_t* __restrict__ slot_off,
+                 const int32_t* __restrict__ slot_row_off, int32_t* __restrict__ pair_row,
+                 int32_t* __restrict__ row_pair, uint4* __restrict__ xp, int32_t* __restrict__ status) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int t = blockIdx.x * kWarpsPerBlock + warp;
   if (t >= T) return;
+  // ---- ranks of this token's K pairs ----
+  int my_rank = -1, my_e = -1;                 // lane j < K ends up holding pair j
+  int64_t cur_seg = -1;
+  int v[kSegPairs / 32];
+  for (int j = 0; j < K; ++j) {
+    const int64_t p = (int64_t)t * K + j;
+    const int64_t seg = p / kSegPairs;
+    if (seg != cur_seg) {                      // (re)load the segment's indices, 8 per lane
+      cur_seg = seg;
+#pragma unroll
+      for (int i = 0; i < kSegPairs / 32; ++i) {
+        const int64_t q = seg * kSegPairs + lane + 32 * i;
+        v[i] = q < R ? topk_idx[q] : -1;
+      }
+    }
+    const int e = topk_idx[p];
+    const int p_local = (int)(p - seg * kSegPairs);
+    int c = 0;
+#pragma unroll
+    for (int i = 0; i < kSegPairs / 32; ++i) c += (lane + 32 * i < p_local && v[i] == e) ? 1 : 0;
+    c = __reduce_add_sync(0xffffffffu, c);
+    if (lane == j) {
+      my_e = e;
+      my_rank = (e >= 0 && e < E) ? seg_base[seg * E + e] + c : -1;
+    }
+  }
+  // ---- replica, slot, row (lane j for pair j) ----
+  int row = -1;
+  if (lane < K && my_rank >= 0) {
+    const long long n = hist[my_e];
+    const int r = replicas[my_e];
+    if (n <= 0 || r < 1 || my_rank >= n) {
+      moegps_report(status, MOEGPS_ERR_HIST_MISMATCH, my_e);
+    } else {
+      const int rho = (int)((((long long)my_rank + 1) * r - 1) / n);   // replica whose range holds the rank
+      const int start = (int)(((long long)rho * n) / r);
+      const int slot = slot_off[my_e] + rho;
+      const long long rr = (slot >= 0 && slot < S) ? (long long)slot_row_off[slot] + (my_rank - start) : -1;
+      if (rr < 0 || rr >= Rcap) {
+        moegps_report(status, MOEGPS_ERR_BAD_INDEX, t);
+      } else {
+        row = (int)rr;
+        pair_row[(int64_t)t * K + lane] = row;
+        row_pair[row] = (int32_t)((int64_t)t * K + lane);
+      }
+    }
+  }
   long long dst[8];
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
-    int row = j < K ? pair_row[(int64_t)t * K + j] : -1;
-    if (row < 0 || row >= Rcap) row = -1;                  // reported by scatter_index; skip here
-    dst[j] = row < 0 ? -1 : (long long)row * chunks;
+    const int rj = __shfl_sync(0xffffffffu, row, j);
+    dst[j] = (j < K && rj >= 0) ? (long long)rj * chunks : -1;
   }
+  // ---- row moves ----
   const uint4* src = x + (int64_t)t * chunks;
   int c = lane;
   for (; c + 96 < chunks; c += 128) {                      // four 16-byte loads in flight per lane
     const uint4 v0 = src[c], v1 = src[c + 32], v2 = src[c + 64], v3 = src[c + 96];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-      if (j < K && dst[j] >= 0) {
+      if (dst[j] >= 0) {
         uint4* d = xp + dst[j];
         d[c] = v0; d[c + 32] = v1; d[c + 64] = v2; d[c + 96] = v3;
       }
     }
   }
   for (; c < chunks; c += 32) {
-    const uint4 v = src[c];
+    const uint4 vv = src[c];
 #pragma unroll
     for (int j = 0; j < 8; ++j)
-      if (j < K && dst[j] >= 0) xp[dst[j] + c] = v;
+      if (dst[j] >= 0) xp[dst[j] + c] = vv;
   }
 }
 
@@ -208,20 +212,15 @@ int moegps_launch_dispatch(moegps_ctx* ctx, const void* x, const int32_t* topk_i
   const int64_t Rcap = moegps_rcap_of(s);
   const int nseg = (int)((R + kSegPairs - 1) / kSegPairs);
   int32_t* seg = static_cast<int32_t*>(workspace);
-  int blocks = (nseg + kWarpsPerBlock - 1) / kWarpsPerBlock;
-  if (blocks < 1) blocks = 1;
-  segment_count_kernel<<<blocks, kThreads, 0, st>>>(topk_idx, R, s.E, seg, nseg, row_pair, Rcap, ctx->d_status);
-  MOEGPS_AFTER_LAUNCH(ctx);
-  scan_offsets_kernel<<<1, 1024, 0, st>>>(seg, nseg, s.E, s.S, s.row_align, hist, replicas, slot_off,
-                                          slot_row_off, ctx->d_status);
+  count_scan_kernel<<<nseg > 0 ? nseg : 1, kScanThreads, 0, st>>>(topk_idx, R, s.E, s.S, s.row_align, seg, nseg,
+                                                                   row_pair, Rcap, hist, replicas, slot_off,
+                                                                   slot_row_off, ctx->d_status);
   MOEGPS_AFTER_LAUNCH(ctx);
   if (R == 0) return MOEGPS_OK;
-  scatter_index_kernel<<<blocks, kThreads, 0, st>>>(topk_idx, R, s.E, s.S, Rcap, seg, nseg, hist, replicas,
-                                                    slot_off, slot_row_off, pair_row, row_pair, ctx->d_status);
-  MOEGPS_AFTER_LAUNCH(ctx);
   const int tblocks = (s.T + kWarpsPerBlock - 1) / kWarpsPerBlock;
-  copy_rows_kernel<<<tblocks, kThreads, 0, st>>>(static_cast<const uint4*>(x), s.T, s.K, s.D / 8, pair_row, Rcap,
-                                                 static_cast<uint4*>(xp));
+  rank_copy_kernel<<<tblocks, kThreads, 0, st>>>(static_cast<const uint4*>(x), s.T, s.K, s.D / 8, topk_idx, R, s.E,
+                                                 s.S, Rcap, seg, hist, replicas, slot_off, slot_row_off, pair_row,
+                                                 row_pair, static_cast<uint4*>(xp), ctx->d_status);
   MOEGPS_AFTER_LAUNCH(ctx);
   return MOEGPS_OK;
 }
