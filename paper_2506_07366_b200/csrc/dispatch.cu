@@ -21,6 +21,7 @@ constexpr int kThreads = kWarpsPerBlock * 32;
 constexpr int kMaxE = 256;
 constexpr int kMaxS = 1024;
 constexpr int kScanThreads = 1024;
+constexpr int kScanSmemBytes = 40 * 1024;   // with the static tables this stays under the 48 KiB default limit
 
 static_assert(kSegPairs == 256, "count_scan assigns one of its first 256 threads to each pair of a segment");
 
@@ -29,11 +30,12 @@ count_scan_kernel(const int32_t* __restrict__ topk_idx, int64_t R, int E, int S,
                   int32_t* seg_cnt, int nseg, int32_t* __restrict__ row_pair, int64_t Rcap,
                   const int32_t* __restrict__ hist, const int32_t* __restrict__ replicas,
                   const int32_t* __restrict__ slot_off, int32_t* __restrict__ slot_row_off,
-                  int32_t* status) {
+                  int e_chunk, int32_t* status) {
   __shared__ int32_t cnt[kMaxE];
   __shared__ int32_t padded[kMaxS];     // rows reserved for each slot (load rounded up to A)
   __shared__ int32_t warp_tot[32];
   __shared__ int is_last;
+  extern __shared__ int32_t scan_mat[];   // [nseg][e_chunk] counts, used by the last CTA only
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int seg = blockIdx.x;
   // padding rows keep -1: fill everything, occupied rows are overwritten by rank_copy
@@ -70,8 +72,35 @@ count_scan_kernel(const int32_t* __restrict__ topk_idx, int64_t R, int E, int S,
   // ---- last CTA only: every segment's counts are now visible ----
   for (int s = tid; s < S; s += blockDim.x) padded[s] = 0;
   __syncthreads();
-  // (a) per expert: exclusive scan of its counts over the segments; lanes stride the segments
-  for (int e = warp; e < E; e += kScanThreads / 32) {
+  // (a) per expert: exclusive scan of its counts over the segments.  The count matrix is pulled
+  // into shared memory `e_chunk` expert columns at a time (coalesced), thread e walks its column,
+  // and the prefix sums are written back (coalesced).
+  for (int e0 = 0; e_chunk > 0 && e0 < E; e0 += e_chunk) {
+    const int ec = min(e_chunk, E - e0);
+    const int n = nseg * ec;
+    for (int i = tid; i < n; i += blockDim.x) {
+      const int g = i / ec, e = i - g * ec;
+      scan_mat[i] = __ldcg(&seg_cnt[(int64_t)g * E + e0 + e]);
+    }
+    __syncthreads();
+    if (tid < ec) {
+      int running = 0;
+      for (int g = 0; g < nseg; ++g) {
+        const int c = scan_mat[g * ec + tid];
+        scan_mat[g * ec + tid] = running;
+        running += c;
+      }
+      if (running != hist[e0 + tid]) moegps_report(status, MOEGPS_ERR_HIST_MISMATCH, e0 + tid);
+    }
+    __syncthreads();
+    for (int i = tid; i < n; i += blockDim.x) {
+      const int g = i / ec, e = i - g * ec;
+      seg_cnt[(int64_t)g * E + e0 + e] = scan_mat[i];
+    }
+    __syncthreads();
+  }
+  // fallback for pair lists too long for shared memory: a warp per expert, lanes stride the segments
+  for (int e = warp; e_chunk == 0 && e < E; e += kScanThreads / 32) {
     int running = 0;
     for (int g0 = 0; g0 < nseg; g0 += 32) {
       const int g = g0 + lane;
@@ -212,9 +241,13 @@ int moegps_launch_dispatch(moegps_ctx* ctx, const void* x, const int32_t* topk_i
   const int64_t Rcap = moegps_rcap_of(s);
   const int nseg = (int)((R + kSegPairs - 1) / kSegPairs);
   int32_t* seg = static_cast<int32_t*>(workspace);
-  count_scan_kernel<<<nseg > 0 ? nseg : 1, kScanThreads, 0, st>>>(topk_idx, R, s.E, s.S, s.row_align, seg, nseg,
-                                                                   row_pair, Rcap, hist, replicas, slot_off,
-                                                                   slot_row_off, ctx->d_status);
+  // expert columns of the count matrix that fit the scan's shared-memory staging (0 = none: fallback path)
+  int e_chunk = nseg > 0 ? kScanSmemBytes / (nseg * (int)sizeof(int32_t)) : s.E;
+  if (e_chunk > s.E) e_chunk = s.E;
+  const size_t scan_smem = (size_t)e_chunk * (nseg > 0 ? nseg : 1) * sizeof(int32_t);
+  count_scan_kernel<<<nseg > 0 ? nseg : 1, kScanThreads, scan_smem, st>>>(
+      topk_idx, R, s.E, s.S, s.row_align, seg, nseg, row_pair, Rcap, hist, replicas, slot_off, slot_row_off, e_chunk,
+      ctx->d_status);
   MOEGPS_AFTER_LAUNCH(ctx);
   if (R == 0) return MOEGPS_OK;
   const int tblocks = (s.T + kWarpsPerBlock - 1) / kWarpsPerBlock;

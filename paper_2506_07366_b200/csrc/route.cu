@@ -23,9 +23,8 @@ using namespace sm100;
 
 constexpr int BM = 128;
 constexpr int BK = 64;
-constexpr int kThreads = 192;
+constexpr int kThreads = 384;   // 12 warps: 2 feed the tensor core, 4 drain TMEM, all 12 reduce and select
 constexpr int kABytes = BM * BK * 2;      // 16 KiB of X per stage
-constexpr int kMaxE = 256;
 
 struct RouteParams {
   int T, D, E, K, gate_mode;
@@ -58,18 +57,54 @@ __device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
   return v;
 }
 
+// One warp per token row: sum the KS partial logits (own and peers' shared memory, fixed order), add
+// the bias, keep the row in registers (lane l holds experts l, l+32, ...) and select.
+template <int NPL>
+__device__ __forceinline__ void reduce_select(const RouteParams& p, const float* partial, uint32_t rank, int m0,
+                                              const float* __restrict__ bias, int32_t* __restrict__ topk_idx,
+                                              float* __restrict__ topk_w, float* __restrict__ logits_out) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rows_per = BM / p.ks;
+  const uint32_t part_u32 = smem_u32(partial);
+  float b[NPL];
+#pragma unroll
+  for (int i = 0; i < NPL; ++i) b[i] = (bias && lane + 32 * i < p.E) ? bias[lane + 32 * i] : 0.f;
+  for (int r = warp; r < rows_per; r += kThreads / 32) {
+    const int row = (int)rank * rows_per + r;
+    const int t = m0 + row;
+    if (t >= p.T) continue;                              // warp-uniform
+    float v[NPL];
+#pragma unroll
+    for (int i = 0; i < NPL; ++i) {
+      const int e = lane + 32 * i;
+      float acc = 0.f;
+      if (e < p.E) {
+        const uint32_t off = part_u32 + (uint32_t)((row * p.part_stride + e) * 4);
+        for (int k = 0; k < p.ks; ++k) acc += ld_cluster_f32(map_to_cta(off, (uint32_t)k));
+      }
+      v[i] = acc + b[i];
+    }
+    if (logits_out) {
+#pragma unroll
+      for (int i = 0; i < NPL; ++i)
+        if (lane + 32 * i < p.E) logits_out[(int64_t)t * p.E + lane + 32 * i] = v[i];
+    }
+    if (topk_idx)
+      warp_topk_gate<NPL>(v, p.E, p.K, p.gate_mode, topk_idx + (int64_t)t * p.K, topk_w + (int64_t)t * p.K);
+  }
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 route_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
              const RouteParams p, const float* __restrict__ bias, int32_t* __restrict__ topk_idx,
              float* __restrict__ topk_w, float* __restrict__ logits_out, int32_t* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  // [ ring (re-used as the partial-logit buffer) | per-warp logit rows | barriers ]
+  // [ ring (re-used as the partial-logit buffer) | barriers ]
   const int part_bytes = BM * p.part_stride * 4;
   const int region0 = p.ring_bytes > part_bytes ? p.ring_bytes : part_bytes;
   float* partial = reinterpret_cast<float*>(smem);
-  float* warp_logit = reinterpret_cast<float*>(smem + region0);                 // [6][kMaxE]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + region0 + 6 * kMaxE * 4);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + region0);
   uint64_t* full = bars;                 // [stages]
   uint64_t* empty = bars + p.stages;     // [stages]
   uint64_t* acc_full = bars + 2 * p.stages;
@@ -134,7 +169,7 @@ route_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
       }
       if (ok && kb_begin < kb_end) mma_commit(acc_full);
     }
-  } else {
+  } else if (warp < 6) {
     // drain this CTA's partial logits: thread = token row, 32 columns per TMEM load
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
@@ -169,30 +204,11 @@ route_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
   cluster_sync_all();           // every CTA's partial is complete and visible cluster-wide
 
   // reduction + selection: CTA `rank` owns rows [rank*rows_per, (rank+1)*rows_per) of the tile
-  {
-    const int rows_per = BM / p.ks;
-    float* mylogit = warp_logit + warp * kMaxE;
-    const uint32_t part_u32 = smem_u32(partial);
-    for (int r = warp; r < rows_per; r += kThreads / 32) {
-      const int row = (int)rank * rows_per + r;
-      const int t = m0 + row;
-      if (t < p.T) {                                     // warp-uniform
-        for (int e = lane; e < p.E; e += 32) {
-          float acc = 0.f;
-          const uint32_t off = part_u32 + (uint32_t)((row * p.part_stride + e) * 4);
-          for (int k = 0; k < p.ks; ++k) acc += ld_cluster_f32(map_to_cta(off, (uint32_t)k));
-          mylogit[e] = acc + (bias ? bias[e] : 0.f);
-        }
-        __syncwarp();
-        if (logits_out)
-          for (int e = lane; e < p.E; e += 32) logits_out[(int64_t)t * p.E + e] = mylogit[e];
-        if (topk_idx)
-          warp_topk_gate<kMaxE / 32>(mylogit, p.E, p.K, p.gate_mode, topk_idx + (int64_t)t * p.K,
-                                     topk_w + (int64_t)t * p.K);
-        __syncwarp();
-      }
-    }
-  }
+  if (p.E <= 32) reduce_select<1>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out);
+  else if (p.E <= 64) reduce_select<2>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out);
+  else if (p.E <= 128) reduce_select<4>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out);
+  else reduce_select<8>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out);
+  __syncwarp();
   cluster_sync_all();           // nobody leaves while a peer may still read its shared memory
   if (warp == 1) {
     tc_fence_after_sync();
@@ -226,7 +242,7 @@ int moegps_launch_route(moegps_ctx* ctx, const void* x, const void* wr, const fl
   p.part_stride = p.e_pad + 1;
   const int part_bytes = BM * p.part_stride * 4;
   const int region0 = p.ring_bytes > part_bytes ? p.ring_bytes : part_bytes;
-  const size_t smem_bytes = 1024 + (size_t)region0 + 6 * kMaxE * 4 + (2 * p.stages + 1) * 8 + 64;
+  const size_t smem_bytes = 1024 + (size_t)region0 + (2 * p.stages + 1) * 8 + 64;
 
   if (!(ctx->rt_valid && ctx->rt_key[0] == x && ctx->rt_key[1] == wr)) {
     ctx->rt_valid = false;

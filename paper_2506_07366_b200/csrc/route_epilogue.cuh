@@ -1,24 +1,32 @@
-// Warp-level epilogue of the router: top-K selection by warp shuffles and the gate weights.
+// Warp-level epilogue of the router: top-K selection across the lanes of a warp and the gate weights.
 #pragma once
 
 #include <math_constants.h>
 
 #include "common.cuh"
 
-// One warp selects the K largest of `logit[0..E)` (shared memory, bias already added) in descending
-// order, equal values by ascending index, and writes indices and gate weights of one token.
-// Lane l owns experts l, l+32, ...; each of the K rounds is a warp arg-max by shuffles, after which
-// the winner is struck from its owner's list.
-template <int kMaxPerLane = 8>
-__device__ __forceinline__ void warp_topk_gate(const float* logit, int E, int K, int gate_mode,
+// Monotone map from fp32 to uint32 (larger float <=> larger key); -0 is folded into +0 first so
+// that equal values have equal keys.
+__device__ __forceinline__ uint32_t route_order_key(float f) {
+  const uint32_t u = __float_as_uint(f + 0.f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float route_key_value(uint32_t k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
+// One warp selects the K largest of E logits, in descending order, equal values by ascending expert
+// index, and lane 0 writes the indices and gate weights of one token.  Lane l holds the logits of
+// experts l, l+32, ... in v[0..NPL).  Each of the K rounds: every lane finds its best remaining
+// entry, a warp-wide max-reduction (redux.sync) finds the winning value, a min-reduction over the
+// lanes that hold it finds the lowest such expert, and its owner strikes it from its list.
+template <int NPL>
+__device__ __forceinline__ void warp_topk_gate(const float (&v)[NPL], int E, int K, int gate_mode,
                                                int32_t* __restrict__ idx_out, float* __restrict__ w_out) {
   const int lane = threadIdx.x & 31;
-  float v[kMaxPerLane];
+  uint32_t key[NPL];
 #pragma unroll
-  for (int i = 0; i < kMaxPerLane; ++i) {
-    const int e = lane + 32 * i;
-    v[i] = e < E ? logit[e] : -CUDART_INF_F;
-  }
+  for (int i = 0; i < NPL; ++i) key[i] = (lane + 32 * i < E) ? route_order_key(v[i]) : 0u;   // 0 < every real key
   unsigned taken = 0;           // bit i: expert lane+32*i already selected
   float sel_v[8];
   int sel_e[8];
@@ -27,30 +35,21 @@ __device__ __forceinline__ void warp_topk_gate(const float* logit, int E, int K,
     sel_v[k] = 0.f;
     sel_e[k] = 0;
     if (k < K) {
-      // local best: strict '>' keeps the lowest index among equal values
-      float bv = -CUDART_INF_F;
+      uint32_t bk = 0u;         // best remaining key of this lane; strict '>' keeps its lowest index
       int be = 0x7fffffff;
 #pragma unroll
-      for (int i = 0; i < kMaxPerLane; ++i) {
-        const int e = lane + 32 * i;
-        if (e < E && !((taken >> i) & 1u) && (be == 0x7fffffff || v[i] > bv)) {
-          bv = v[i];
-          be = e;
+      for (int i = 0; i < NPL; ++i) {
+        const bool live = (lane + 32 * i < E) && !((taken >> i) & 1u);
+        if (live && (be == 0x7fffffff || key[i] > bk)) {
+          bk = key[i];
+          be = lane + 32 * i;
         }
       }
-#pragma unroll
-      for (int m = 16; m >= 1; m >>= 1) {
-        const float ov = __shfl_xor_sync(0xffffffffu, bv, m);
-        const int oe = __shfl_xor_sync(0xffffffffu, be, m);
-        const bool other_valid = oe != 0x7fffffff, mine_valid = be != 0x7fffffff;
-        if (other_valid && (!mine_valid || ov > bv || (ov == bv && oe < be))) {
-          bv = ov;
-          be = oe;
-        }
-      }
-      sel_v[k] = bv;
-      sel_e[k] = be;
-      if ((be & 31) == lane) taken |= 1u << (be >> 5);
+      const uint32_t wk = __reduce_max_sync(0xffffffffu, be == 0x7fffffff ? 0u : bk);
+      const uint32_t we = __reduce_min_sync(0xffffffffu, (be != 0x7fffffff && bk == wk) ? (uint32_t)be : 0xffffffffu);
+      sel_v[k] = route_key_value(wk);
+      sel_e[k] = (int)we;
+      if ((int)(we & 31u) == lane) taken |= 1u << (we >> 5);
     }
   }
   if (lane == 0) {
