@@ -72,7 +72,8 @@ _LIB = None
 
 
 def library_path() -> str:
-    return _build.LIB_PATH
+    """The in-tree build, unless MOEGPS_LIBRARY names another build of the same library."""
+    return os.environ.get("MOEGPS_LIBRARY") or _build.LIB_PATH
 
 
 def _lib():

@@ -77,25 +77,33 @@ count_scan_kernel(const int32_t* __restrict__ topk_idx, int64_t R, int E, int S,
   // and the prefix sums are written back (coalesced).
   for (int e0 = 0; e_chunk > 0 && e0 < E; e0 += e_chunk) {
     const int ec = min(e_chunk, E - e0);
+    const int ecp = ec | 1;                     // odd row stride: a column walk hits distinct banks
     const int n = nseg * ec;
     for (int i = tid; i < n; i += blockDim.x) {
       const int g = i / ec, e = i - g * ec;
-      scan_mat[i] = __ldcg(&seg_cnt[(int64_t)g * E + e0 + e]);
+      scan_mat[g * ecp + e] = __ldcg(&seg_cnt[(int64_t)g * E + e0 + e]);
     }
     __syncthreads();
-    if (tid < ec) {
+    for (int c = warp; c < ec; c += kScanThreads / 32) {      // one warp per expert column
       int running = 0;
-      for (int g = 0; g < nseg; ++g) {
-        const int c = scan_mat[g * ec + tid];
-        scan_mat[g * ec + tid] = running;
-        running += c;
+      for (int g0 = 0; g0 < nseg; g0 += 32) {
+        const int g = g0 + lane;
+        const int v = g < nseg ? scan_mat[g * ecp + c] : 0;
+        int incl = v;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          const int o = __shfl_up_sync(0xffffffffu, incl, d);
+          if (lane >= d) incl += o;
+        }
+        if (g < nseg) scan_mat[g * ecp + c] = running + incl - v;
+        running += __shfl_sync(0xffffffffu, incl, 31);
       }
-      if (running != hist[e0 + tid]) moegps_report(status, MOEGPS_ERR_HIST_MISMATCH, e0 + tid);
+      if (lane == 0 && running != hist[e0 + c]) moegps_report(status, MOEGPS_ERR_HIST_MISMATCH, e0 + c);
     }
     __syncthreads();
     for (int i = tid; i < n; i += blockDim.x) {
       const int g = i / ec, e = i - g * ec;
-      seg_cnt[(int64_t)g * E + e0 + e] = scan_mat[i];
+      seg_cnt[(int64_t)g * E + e0 + e] = scan_mat[g * ecp + e];
     }
     __syncthreads();
   }
@@ -124,9 +132,13 @@ count_scan_kernel(const int32_t* __restrict__ topk_idx, int64_t R, int E, int S,
     if (r < 1 || so < 0 || so + r > S || n < 0) {
       moegps_report(status, MOEGPS_ERR_BAD_INDEX, tid);
     } else {
-      for (int rho = 0; rho < r; ++rho) {
-        const int load = (int)(((rho + 1) * n) / r - (rho * n) / r);
-        padded[so + rho] = (load + A - 1) / A * A;
+      // floor(rho n / r) = rho q + floor(rho m / r) with n = q r + m: one division, then 32-bit work
+      const int q = (int)(n / r), m = (int)(n - (long long)q * r);
+      int prev = 0;
+      for (int rho = 1; rho <= r; ++rho) {
+        const int start = rho * q + (rho * m) / r;     // rho, m < r <= 1024
+        padded[so + rho - 1] = (start - prev + A - 1) / A * A;
+        prev = start;
       }
     }
   }
@@ -242,9 +254,10 @@ int moegps_launch_dispatch(moegps_ctx* ctx, const void* x, const int32_t* topk_i
   const int nseg = (int)((R + kSegPairs - 1) / kSegPairs);
   int32_t* seg = static_cast<int32_t*>(workspace);
   // expert columns of the count matrix that fit the scan's shared-memory staging (0 = none: fallback path)
-  int e_chunk = nseg > 0 ? kScanSmemBytes / (nseg * (int)sizeof(int32_t)) : s.E;
+  int e_chunk = nseg > 0 ? kScanSmemBytes / (nseg * (int)sizeof(int32_t)) - 1 : s.E;   // -1: odd row stride
   if (e_chunk > s.E) e_chunk = s.E;
-  const size_t scan_smem = (size_t)e_chunk * (nseg > 0 ? nseg : 1) * sizeof(int32_t);
+  if (e_chunk < 0) e_chunk = 0;
+  const size_t scan_smem = e_chunk > 0 ? (size_t)(e_chunk | 1) * (nseg > 0 ? nseg : 1) * sizeof(int32_t) : 0;
   count_scan_kernel<<<nseg > 0 ? nseg : 1, kScanThreads, scan_smem, st>>>(
       topk_idx, R, s.E, s.S, s.row_align, seg, nseg, row_pair, Rcap, hist, replicas, slot_off, slot_row_off, e_chunk,
       ctx->d_status);

@@ -18,8 +18,15 @@ using namespace sm100;
 
 constexpr int BM = 128;            // rows per tile
 constexpr int BNACC = 256;         // accumulator columns per tile
-constexpr int BK = 64;             // K elements per stage: 128 bytes = one swizzle row
-constexpr int kStages = 4;
+#ifndef MOEGPS_FFN_BK
+#define MOEGPS_FFN_BK 64
+#endif
+// K elements per stage = one swizzle row of BK*2 bytes.  Measured on B200: 64 (128-byte rows, 4
+// stages of 48 KiB) beats 32 (64-byte rows, 8 stages of 24 KiB) by about 25 %: TMA moves 128-byte
+// rows far more efficiently, which outweighs the deeper ring.
+constexpr int BK = MOEGPS_FFN_BK;
+constexpr int kRowBytes = BK * 2;
+constexpr int kStages = 256 / BK;  // 192 KiB of ring either way
 constexpr int kABytes = BM * BK * 2;
 constexpr int kBHalfBytes = 128 * BK * 2;
 constexpr int kStageBytes = kABytes + 2 * kBHalfBytes;       // 48 KiB
@@ -42,7 +49,7 @@ struct TileCoord {
   int expert;
 };
 
-__device__ __forceinline__ TileCoord decode_tile(const Tables& tb, int S, int tile, int n_tiles) {
+__device__ __forceinline__ TileCoord decode_tile_rows(const Tables& tb, int S, int tile, int n_tiles, int tile_rows) {
   int lo = 0, hi = S;                 // find s with tile_base[s] <= tile < tile_base[s+1]
   while (hi - lo > 1) {
     const int mid = (lo + hi) >> 1;
@@ -53,15 +60,65 @@ __device__ __forceinline__ TileCoord decode_tile(const Tables& tb, int S, int ti
   const int mt = (tb.tile_base[s + 1] - tb.tile_base[s]) / n_tiles;   // row tiles of this slot
   TileCoord c;
   c.n_tile = local / mt;
-  c.m0 = tb.row_off[s] + (local % mt) * BM;
+  c.m0 = tb.row_off[s] + (local % mt) * tile_rows;
   c.row_end = tb.row_off[s + 1];
   c.expert = tb.expert[s];
   return c;
 }
 
+__device__ __forceinline__ TileCoord decode_tile(const Tables& tb, int S, int tile, int n_tiles) {
+  return decode_tile_rows(tb, S, tile, n_tiles, BM);
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+// Epilogue of one tile for one thread (= one accumulator row): TMEM -> registers -> bf16 -> global.
+// kSwiGLU: columns [0,128) are the gate and [128,256) the up projection; 128 outputs silu(g)*u.
+template <bool kSwiGLU>
+__device__ __forceinline__ void drain_tile(uint32_t taddr, bool row_ok, __nv_bfloat16* orow, int col0, int n_dim) {
+if constexpr (kSwiGLU) {
+#pragma unroll 1
+  for (int c0 = 0; c0 < 128; c0 += 32) {
+    uint32_t g[32], u[32];
+    tmem_ld32(taddr + c0, g);
+    tmem_ld32(taddr + 128 + c0, u);
+    tmem_ld_wait();
+    uint32_t o[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
+      // silu(g) * u with the fast reciprocal (2 ulp): the result is rounded to bf16 right after
+      const float h0 = __fdividef(g0, 1.f + __expf(-g0)) * __uint_as_float(u[2 * i]);
+      const float h1 = __fdividef(g1, 1.f + __expf(-g1)) * __uint_as_float(u[2 * i + 1]);
+      o[i] = pack_bf16(h0, h1);
+    }
+    if (row_ok) {
+#pragma unroll
+      for (int v = 0; v < 4; ++v)
+        if (col0 + c0 + 8 * v + 8 <= n_dim)
+          *reinterpret_cast<uint4*>(orow + c0 + 8 * v) = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
+    }
+  }
+} else {
+#pragma unroll 1
+  for (int c0 = 0; c0 < 256; c0 += 32) {
+    uint32_t a[32];
+    tmem_ld32(taddr + c0, a);
+    tmem_ld_wait();
+    uint32_t o[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) o[i] = pack_bf16(__uint_as_float(a[2 * i]), __uint_as_float(a[2 * i + 1]));
+    if (row_ok) {
+#pragma unroll
+      for (int v = 0; v < 4; ++v)
+        if (col0 + c0 + 8 * v + 8 <= n_dim)
+          *reinterpret_cast<uint4*>(orow + c0 + 8 * v) = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
+    }
+  }
+}
 }
 
 // kSwiGLU = true : out[row, n_tile*128 + c] = silu(acc[c]) * acc[128 + c],  c < 128
@@ -166,8 +223,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
           if (!mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
           tc_fence_after_sync();
           const uint32_t sa = smem_u32(stage_mem + (size_t)stage * kStageBytes);
-          const uint64_t da = smem_desc_k_sw128(sa);
-          const uint64_t db = smem_desc_k_sw128(sa + kABytes);
+          const uint64_t da = smem_desc_k<kRowBytes>(sa);
+          const uint64_t db = smem_desc_k<kRowBytes>(sa + kABytes);
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k)      // 16 bf16 = 32 bytes per MMA along K
             mma_bf16(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb | k) != 0);
@@ -190,52 +247,14 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
       const TileCoord tc = decode_tile(tb, S, tile, n_tiles);
-      if (!mbar_wait(&acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
+      if (!mbar_wait(&acc_full[acc], acc_phase, abort_flag, 256)) { ok = false; break; }
       tc_fence_after_sync();
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * BNACC;
       const int row = tc.m0 + row_in_tile;
       const bool row_ok = row < tc.row_end;
       const int col0 = tc.n_tile * cols_per_tile;
       __nv_bfloat16* orow = out + (size_t)row * n_dim + col0;
-      if constexpr (kSwiGLU) {
-#pragma unroll 1
-        for (int c0 = 0; c0 < 128; c0 += 32) {
-          uint32_t g[32], u[32];
-          tmem_ld32(taddr + c0, g);
-          tmem_ld32(taddr + 128 + c0, u);
-          tmem_ld_wait();
-          uint32_t o[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
-            const float h0 = g0 / (1.f + __expf(-g0)) * __uint_as_float(u[2 * i]);
-            const float h1 = g1 / (1.f + __expf(-g1)) * __uint_as_float(u[2 * i + 1]);
-            o[i] = pack_bf16(h0, h1);
-          }
-          if (row_ok) {
-#pragma unroll
-            for (int v = 0; v < 4; ++v)
-              if (col0 + c0 + 8 * v + 8 <= n_dim)
-                *reinterpret_cast<uint4*>(orow + c0 + 8 * v) = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
-          }
-        }
-      } else {
-#pragma unroll 1
-        for (int c0 = 0; c0 < 256; c0 += 32) {
-          uint32_t a[32];
-          tmem_ld32(taddr + c0, a);
-          tmem_ld_wait();
-          uint32_t o[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) o[i] = pack_bf16(__uint_as_float(a[2 * i]), __uint_as_float(a[2 * i + 1]));
-          if (row_ok) {
-#pragma unroll
-            for (int v = 0; v < 4; ++v)
-              if (col0 + c0 + 8 * v + 8 <= n_dim)
-                *reinterpret_cast<uint4*>(orow + c0 + 8 * v) = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
-          }
-        }
-      }
+      drain_tile<kSwiGLU>(taddr, row_ok, orow, col0, n_dim);
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(&acc_empty[acc]);
@@ -273,30 +292,39 @@ EncodeTiledFn get_encode_fn() {
 
 }  // namespace
 
-// bf16 [rows, cols] row-major; box = 64 columns x box_rows rows, 128-byte swizzle, zero fill outside.
-bool moegps_make_tmap_2d(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+namespace {
+CUtensorMapSwizzle swizzle_for(uint32_t box_cols) {   // swizzle span = the box's row length in bytes
+  return box_cols == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : (box_cols == 32 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                                                      : CU_TENSOR_MAP_SWIZZLE_32B);
+}
+}  // namespace
+
+// bf16 [rows, cols] row-major; box = box_cols (64, 32 or 16) columns x box_rows rows, swizzle span =
+// the box's row length, zero fill outside.
+bool moegps_make_tmap_2d(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                         uint32_t box_cols) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[2] = {cols, rows};
   const cuuint64_t strides[1] = {cols * 2};
-  const cuuint32_t box[2] = {64, box_rows};
+  const cuuint32_t box[2] = {box_cols, box_rows};
   const cuuint32_t estr[2] = {1, 1};
   return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(box_cols), CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// bf16 [batch, rows, cols]; box = 64 columns x box_rows rows x 1 batch entry.
+// bf16 [batch, rows, cols]; box = box_cols columns x box_rows rows x 1 batch entry.
 bool moegps_make_tmap_3d(CUtensorMap* tm, const void* base, uint64_t batch, uint64_t rows, uint64_t cols,
-                         uint32_t box_rows) {
+                         uint32_t box_rows, uint32_t box_cols) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[3] = {cols, rows, batch};
   const cuuint64_t strides[2] = {cols * 2, rows * cols * 2};
-  const cuuint32_t box[3] = {64, box_rows, 1};
+  const cuuint32_t box[3] = {box_cols, box_rows, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
   return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(box_cols), CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -326,9 +354,9 @@ int moegps_launch_ffn_gate_up(moegps_ctx* ctx, const void* xp, const int32_t* sl
   const uint64_t rcap = (uint64_t)moegps_rcap_of(s);
   if (!(ctx->tm1_valid && ctx->tm_key1[0] == xp && ctx->tm_key1[1] == w_gate && ctx->tm_key1[2] == w_up)) {
     ctx->tm1_valid = false;
-    if (!(moegps_make_tmap_2d(&ctx->tm_xp, xp, rcap, s.D, BM) &&
-          moegps_make_tmap_3d(&ctx->tm_w1, w_gate, s.E, s.F, s.D, 128) &&
-          moegps_make_tmap_3d(&ctx->tm_w3, w_up, s.E, s.F, s.D, 128)))
+    if (!(moegps_make_tmap_2d(&ctx->tm_xp, xp, rcap, s.D, BM, BK) &&
+          moegps_make_tmap_3d(&ctx->tm_w1, w_gate, s.E, s.F, s.D, 128, BK) &&
+          moegps_make_tmap_3d(&ctx->tm_w3, w_up, s.E, s.F, s.D, 128, BK)))
       return tmap_failed(ctx);
     ctx->tm_key1[0] = xp; ctx->tm_key1[1] = w_gate; ctx->tm_key1[2] = w_up;
     ctx->tm1_valid = true;
@@ -348,8 +376,8 @@ int moegps_launch_ffn_down(moegps_ctx* ctx, const void* h_ws, const int32_t* slo
   const uint64_t rcap = (uint64_t)moegps_rcap_of(s);
   if (!(ctx->tm2_valid && ctx->tm_key2[0] == h_ws && ctx->tm_key2[1] == w_down)) {
     ctx->tm2_valid = false;
-    if (!(moegps_make_tmap_2d(&ctx->tm_h, h_ws, rcap, s.F, BM) &&
-          moegps_make_tmap_3d(&ctx->tm_w2, w_down, s.E, s.D, s.F, 128)))
+    if (!(moegps_make_tmap_2d(&ctx->tm_h, h_ws, rcap, s.F, BM, BK) &&
+          moegps_make_tmap_3d(&ctx->tm_w2, w_down, s.E, s.D, s.F, 128, BK)))
       return tmap_failed(ctx);
     ctx->tm_key2[0] = h_ws; ctx->tm_key2[1] = w_down;
     ctx->tm2_valid = true;

@@ -45,8 +45,7 @@ __global__ void __launch_bounds__(kPlanThreads)
 plan_kernel(const int32_t* __restrict__ pred, int E, int S, int c_max, int32_t* __restrict__ replicas,
             int32_t* __restrict__ slot_off, int32_t* __restrict__ slot_expert, int32_t* __restrict__ bound,
             int32_t* __restrict__ status) {
-  __shared__ Cand warp_c[kPlanThreads / 32];
-  __shared__ Cand winner;
+  __shared__ int plan_r[kPlanThreads];
   __shared__ int warp_sum[kPlanThreads / 32];
   __shared__ int warp_max[kPlanThreads / 32];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -59,27 +58,41 @@ plan_kernel(const int32_t* __restrict__ pred, int E, int S, int c_max, int32_t* 
     n = v < 0 ? 0 : v;
     r = 1;
   }
-  for (int round = 0; round < S - E; ++round) {
-    Cand c;
-    c.n = (mine && (c_max <= 0 || r < c_max)) ? n : -1;
-    c.r = r;
-    c.e = tid;
-    c = warp_best(c);
-    if (lane == 0) warp_c[warp] = c;
-    __syncthreads();
-    if (warp == 0) {
-      Cand d;
-      d.n = -1; d.r = 0; d.e = kPlanThreads + lane;
-      if (lane < kPlanThreads / 32) d = warp_c[lane];
-      d = warp_best(d);
-      if (lane == 0) winner = d;
+  // The S-E rounds run on warp 0 alone (no block barriers inside the loop): lane l keeps experts
+  // l, l+32, ... in registers, picks its best candidate, and a shuffle butterfly picks the winner.
+  if (warp == 0) {
+    constexpr int kPerLane = kPlanThreads / 32;
+    long long ln[kPerLane];
+    int lr[kPerLane];
+#pragma unroll
+    for (int i = 0; i < kPerLane; ++i) {
+      const int e = lane + 32 * i;
+      const int v = e < E ? pred[e] : 0;
+      ln[i] = e < E ? (v < 0 ? 0 : v) : -1;
+      lr[i] = e < E ? 1 : 0;
     }
-    __syncthreads();
-    const Cand w = winner;
-    if (w.n < 0) break;            // nobody may take another copy: the remaining slots stay empty
-    if (w.e == tid) r += 1;
-    // `winner`/`warp_c` are rewritten only after the next round's first barrier
+    for (int round = 0; round < S - E; ++round) {
+      Cand c;
+      c.n = -1; c.r = 0; c.e = kPlanThreads + lane;
+#pragma unroll
+      for (int i = 0; i < kPerLane; ++i) {
+        Cand d;
+        d.n = (ln[i] >= 0 && (c_max <= 0 || lr[i] < c_max)) ? ln[i] : -1;
+        d.r = lr[i];
+        d.e = lane + 32 * i;
+        if (better(d, c)) c = d;
+      }
+      c = warp_best(c);
+      if (c.n < 0) break;          // nobody may take another copy: the remaining slots stay empty
+#pragma unroll
+      for (int i = 0; i < kPerLane; ++i)
+        if (c.e == lane + 32 * i) lr[i] += 1;
+    }
+#pragma unroll
+    for (int i = 0; i < kPerLane; ++i) plan_r[lane + 32 * i] = lr[i];
   }
+  __syncthreads();
+  if (mine) r = plan_r[tid];
   // slot_off = exclusive prefix sum of r
   int incl = mine ? r : 0;
 #pragma unroll

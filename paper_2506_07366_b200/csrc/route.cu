@@ -15,7 +15,8 @@
 #include "route_epilogue.cuh"
 #include "sm100.cuh"
 
-bool moegps_make_tmap_2d(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+bool moegps_make_tmap_2d(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                         uint32_t box_cols);
 
 namespace {
 
@@ -37,35 +38,26 @@ struct RouteParams {
   int part_stride;  // floats per row of the partial-logit buffer (e_pad + 1: conflict-free)
 };
 
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// Address of `local_smem_addr` in the shared memory of CTA `rank` of this cluster.
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_smem_addr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_smem_addr), "r"(rank));
-  return r;
-}
+// volatile keeps these loads behind the cluster barrier (also a volatile asm) and in program
+// order; callers issue a batch of them before using any result so that they overlap.
 __device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
   float v;
-  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr));
   return v;
 }
 
-// One warp per token row: sum the KS partial logits (own and peers' shared memory, fixed order), add
-// the bias, keep the row in registers (lane l holds experts l, l+32, ...) and select.
-template <int NPL>
+// One warp per token row: fetch the KS partial logits of the row (own and peers' shared memory),
+// sum them in slice order, add the bias, keep the row in registers (lane l holds experts l,
+// l+32, ...) and select.
+template <int NPL, int KS>
 __device__ __forceinline__ void reduce_select(const RouteParams& p, const float* partial, uint32_t rank, int m0,
                                               const float* __restrict__ bias, int32_t* __restrict__ topk_idx,
                                               float* __restrict__ topk_w, float* __restrict__ logits_out) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int rows_per = BM / p.ks;
-  const uint32_t part_u32 = smem_u32(partial);
+  constexpr int rows_per = BM / KS;
+  uint32_t peer[KS];
+#pragma unroll
+  for (int k = 0; k < KS; ++k) peer[k] = map_to_cta(smem_u32(partial), (uint32_t)k);
   float b[NPL];
 #pragma unroll
   for (int i = 0; i < NPL; ++i) b[i] = (bias && lane + 32 * i < p.E) ? bias[lane + 32 * i] : 0.f;
@@ -73,15 +65,20 @@ __device__ __forceinline__ void reduce_select(const RouteParams& p, const float*
     const int row = (int)rank * rows_per + r;
     const int t = m0 + row;
     if (t >= p.T) continue;                              // warp-uniform
-    float v[NPL];
+    float raw[NPL][KS];
 #pragma unroll
     for (int i = 0; i < NPL; ++i) {
       const int e = lane + 32 * i;
+      const uint32_t off = (uint32_t)((row * p.part_stride + (e < p.E ? e : 0)) * 4);
+#pragma unroll
+      for (int k = 0; k < KS; ++k) raw[i][k] = ld_cluster_f32(peer[k] + off);
+    }
+    float v[NPL];
+#pragma unroll
+    for (int i = 0; i < NPL; ++i) {
       float acc = 0.f;
-      if (e < p.E) {
-        const uint32_t off = part_u32 + (uint32_t)((row * p.part_stride + e) * 4);
-        for (int k = 0; k < p.ks; ++k) acc += ld_cluster_f32(map_to_cta(off, (uint32_t)k));
-      }
+#pragma unroll
+      for (int k = 0; k < KS; ++k) acc += raw[i][k];
       v[i] = acc + b[i];
     }
     if (logits_out) {
@@ -204,10 +201,18 @@ route_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
   cluster_sync_all();           // every CTA's partial is complete and visible cluster-wide
 
   // reduction + selection: CTA `rank` owns rows [rank*rows_per, (rank+1)*rows_per) of the tile
-  if (p.E <= 32) reduce_select<1>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out);
-  else if (p.E <= 64) reduce_select<2>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out);
-  else if (p.E <= 128) reduce_select<4>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out);
-  else reduce_select<8>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out);
+#define MOEGPS_ROUTE_SELECT(NPL)                                                                          \
+  switch (p.ks) {                                                                                         \
+    case 1: reduce_select<NPL, 1>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out); break;       \
+    case 2: reduce_select<NPL, 2>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out); break;       \
+    case 4: reduce_select<NPL, 4>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out); break;       \
+    default: reduce_select<NPL, 8>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out); break;      \
+  }
+  if (p.E <= 32) { MOEGPS_ROUTE_SELECT(1) }
+  else if (p.E <= 64) { MOEGPS_ROUTE_SELECT(2) }
+  else if (p.E <= 128) { MOEGPS_ROUTE_SELECT(4) }
+  else { MOEGPS_ROUTE_SELECT(8) }
+#undef MOEGPS_ROUTE_SELECT
   __syncwarp();
   cluster_sync_all();           // nobody leaves while a peer may still read its shared memory
   if (warp == 1) {
@@ -246,8 +251,8 @@ int moegps_launch_route(moegps_ctx* ctx, const void* x, const void* wr, const fl
 
   if (!(ctx->rt_valid && ctx->rt_key[0] == x && ctx->rt_key[1] == wr)) {
     ctx->rt_valid = false;
-    if (!(moegps_make_tmap_2d(&ctx->tm_rx, x, (uint64_t)s.T, (uint64_t)s.D, BM) &&
-          moegps_make_tmap_2d(&ctx->tm_rw, wr, (uint64_t)s.E, (uint64_t)s.D, (uint32_t)p.e_pad))) {
+    if (!(moegps_make_tmap_2d(&ctx->tm_rx, x, (uint64_t)s.T, (uint64_t)s.D, BM, BK) &&
+          moegps_make_tmap_2d(&ctx->tm_rw, wr, (uint64_t)s.E, (uint64_t)s.D, (uint32_t)p.e_pad, BK))) {
       ctx->last_cuda_error = (int)cudaErrorInvalidValue;
       return MOEGPS_ERR_CUDA;
     }

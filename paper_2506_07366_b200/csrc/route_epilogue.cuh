@@ -52,25 +52,25 @@ __device__ __forceinline__ void warp_topk_gate(const float (&v)[NPL], int E, int
       if ((int)(we & 31u) == lane) taken |= 1u << (we >> 5);
     }
   }
-  if (lane == 0) {
-    float g[8];
-    float sum = 0.f;
+  // every lane knows all K selections; lane k < K computes and stores the k-th gate weight
+  float myv = 0.f;
+  int mye = 0;
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      g[k] = 0.f;
-      if (k < K) {
-        // sel_v[0] is the largest logit
-        g[k] = gate_mode == 0 ? __expf(sel_v[k] - sel_v[0]) : 1.f / (1.f + __expf(-sel_v[k]));
-        sum += g[k];
-      }
+  for (int k = 0; k < 8; ++k) {
+    if (k < K && lane == k) {
+      myv = sel_v[k];
+      mye = sel_e[k];
     }
-    const float inv = 1.f / sum;
-#pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      if (k < K) {
-        idx_out[k] = sel_e[k];
-        w_out[k] = g[k] * inv;
-      }
-    }
+  }
+  float g = 0.f;
+  if (lane < K) g = gate_mode == 0 ? __expf(myv - sel_v[0]) /* sel_v[0] is the largest logit */
+                                   : 1.f / (1.f + __expf(-myv));
+  float sum = g;                 // lanes K..7 contribute 0; K <= 8
+  sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+  sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+  sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+  if (lane < K) {
+    idx_out[lane] = mye;
+    w_out[lane] = g / sum;
   }
 }

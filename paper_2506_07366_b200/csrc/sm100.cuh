@@ -45,12 +45,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // polled too, so that one role giving up makes the others give up promptly.
 constexpr long long kWaitLimitCycles = 2000000000ll;
 
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+// `sleep_ns` > 0 makes the waiter back off between polls: waits that are expected to be long
+// (an epilogue warp waiting for a whole main loop) should not burn issue slots and power that the
+// tensor pipe needs; latency-critical waits pass 0.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          unsigned sleep_ns = 0) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   uint32_t spins = 0;
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
+    if (sleep_ns) __nanosleep(sleep_ns);
     if ((++spins & 63u) == 0) {
       if (*abort_flag) return false;
       if (clock64() - t0 > kWaitLimitCycles) {
@@ -107,15 +112,21 @@ __device__ __forceinline__ void tc_fence_after_sync() {
 // with the 128-byte swizzle TMA applies: 8-row groups are 1024 bytes apart, the tile base is
 // 1024-byte aligned.  Advancing along K inside the 128-byte row is done by adding the byte offset
 // (>> 4) to the start-address field.
-__device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t smem_addr) {
+// The same for rows of kRowBytes = 128, 64 or 32 bytes (swizzle span = row length; 8-row groups
+// are 8*kRowBytes apart and the tile base is aligned to that).
+template <int kRowBytes>
+__device__ __forceinline__ uint64_t smem_desc_k(uint32_t smem_addr) {
+  static_assert(kRowBytes == 128 || kRowBytes == 64 || kRowBytes == 32, "swizzle span");
+  constexpr uint64_t layout = kRowBytes == 128 ? 2 : (kRowBytes == 64 ? 4 : 6);
   uint64_t d = 0;
   d |= (uint64_t)((smem_addr & 0x3ffffu) >> 4);          // start address, bits [0,14)
   d |= (uint64_t)1 << 16;                                // leading byte offset (unused with swizzle), bits [16,30)
-  d |= (uint64_t)(1024 >> 4) << 32;                      // stride byte offset: 8 rows x 128 B, bits [32,46)
+  d |= (uint64_t)((8 * kRowBytes) >> 4) << 32;           // stride byte offset: 8 rows, bits [32,46)
   d |= (uint64_t)1 << 46;                                // descriptor version for this architecture
-  d |= (uint64_t)2 << 61;                                // layout: 128-byte swizzle
+  d |= layout << 61;                                     // layout: swizzle mode
   return d;
 }
+__device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t smem_addr) { return smem_desc_k<128>(smem_addr); }
 
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, tile M x N.
 __host__ __device__ constexpr uint32_t idesc_bf16_f32(int M, int N) {
@@ -159,4 +170,19 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// ----------------------------------------------------------------------------------- clusters
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cluster address of `local_smem_addr` in the shared memory of CTA `rank` of this cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_smem_addr), "r"(rank));
+  return r;
+}
 }  // namespace sm100

@@ -239,6 +239,11 @@ FFN_CASES = [
     (700, 128, 1408, 16, 4, 20, 128, 1.2),     # several row tiles per slot, F = 11 x 128
     (64, 64, 64, 32, 8, 40, 128, 1.0),         # many almost-empty slots
     (5, 2048, 256, 2, 1, 2, 128, 0.0),         # long K loop, a handful of rows
+    # long slots: many row tiles per slot, more tiles than CTAs (several rounds of the persistent loop)
+    (1500, 256, 384, 2, 2, 3, 128, 0.5),
+    (1500, 256, 384, 2, 2, 3, 1, 0.5),         # unaligned slots: row tiles straddle slot ends
+    (3000, 128, 256, 4, 1, 4, 128, 1.5),       # one hot slot with many row tiles, cold ones with one
+    (1100, 200, 328, 2, 1, 2, 128, 0.0),       # ragged K and N tails with several row tiles
 ]
 
 
