@@ -30,7 +30,7 @@ constexpr int kStages = 256 / BK;  // 192 KiB of ring either way
 constexpr int kABytes = BM * BK * 2;
 constexpr int kBHalfBytes = 128 * BK * 2;
 constexpr int kStageBytes = kABytes + 2 * kBHalfBytes;       // 48 KiB
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;      // producer warp, MMA warp, 8 epilogue warps (two per TMEM lane quarter)
 constexpr int kMaxS = 1024;
 constexpr int kTmemCols = 512;
 
@@ -75,13 +75,24 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 
+// silu(g) = g / (1 + exp(-g)) = g * (0.5 + 0.5 tanh(g / 2)), with the hardware tanh approximation
+// (relative error about 2^-11; the product is rounded to bf16, 2^-9, right after).
+__device__ __forceinline__ float silu_fast(float g) {
+  float t;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(0.5f * g));
+  return g * fmaf(0.5f, t, 0.5f);
+}
+
 // Epilogue of one tile for one thread (= one accumulator row): TMEM -> registers -> bf16 -> global.
 // kSwiGLU: columns [0,128) are the gate and [128,256) the up projection; 128 outputs silu(g)*u.
+// `half` (0 or 1) selects which half of the tile's output columns this warp drains: two warps share
+// each quarter of the TMEM lanes.
 template <bool kSwiGLU>
-__device__ __forceinline__ void drain_tile(uint32_t taddr, bool row_ok, __nv_bfloat16* orow, int col0, int n_dim) {
+__device__ __forceinline__ void drain_tile(uint32_t taddr, bool row_ok, __nv_bfloat16* orow, int col0, int n_dim,
+                                           int half) {
 if constexpr (kSwiGLU) {
 #pragma unroll 1
-  for (int c0 = 0; c0 < 128; c0 += 32) {
+  for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 32) {
     uint32_t g[32], u[32];
     tmem_ld32(taddr + c0, g);
     tmem_ld32(taddr + 128 + c0, u);
@@ -90,9 +101,8 @@ if constexpr (kSwiGLU) {
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
       const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
-      // silu(g) * u with the fast reciprocal (2 ulp): the result is rounded to bf16 right after
-      const float h0 = __fdividef(g0, 1.f + __expf(-g0)) * __uint_as_float(u[2 * i]);
-      const float h1 = __fdividef(g1, 1.f + __expf(-g1)) * __uint_as_float(u[2 * i + 1]);
+      const float h0 = silu_fast(g0) * __uint_as_float(u[2 * i]);
+      const float h1 = silu_fast(g1) * __uint_as_float(u[2 * i + 1]);
       o[i] = pack_bf16(h0, h1);
     }
     if (row_ok) {
@@ -104,7 +114,7 @@ if constexpr (kSwiGLU) {
   }
 } else {
 #pragma unroll 1
-  for (int c0 = 0; c0 < 256; c0 += 32) {
+  for (int c0 = 128 * half; c0 < 128 * half + 128; c0 += 32) {
     uint32_t a[32];
     tmem_ld32(taddr + c0, a);
     tmem_ld_wait();
@@ -152,7 +162,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
   for (int s = threadIdx.x; s < S; s += kThreads) tb.expert[s] = slot_expert[s];
   if (threadIdx.x == 0) {
     for (int i = 0; i < kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 4); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 8); }
     *abort_flag = 0;
     fence_mbar_init();
     prefetch_tensormap(&tm_a);
@@ -241,6 +251,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     }
   } else {
     const int quarter = warp & 3;                 // TMEM lanes this warp may read
+    const int half = (warp - 2) >> 2;             // which half of the output columns it drains
     const int row_in_tile = quarter * 32 + lane;
     int acc = 0;
     uint32_t acc_phase = 0;
@@ -254,7 +265,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
       const bool row_ok = row < tc.row_end;
       const int col0 = tc.n_tile * cols_per_tile;
       __nv_bfloat16* orow = out + (size_t)row * n_dim + col0;
-      drain_tile<kSwiGLU>(taddr, row_ok, orow, col0, n_dim);
+      drain_tile<kSwiGLU>(taddr, row_ok, orow, col0, n_dim, half);
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(&acc_empty[acc]);
