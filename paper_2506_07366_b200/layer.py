@@ -45,19 +45,21 @@ class MoeLayer:
                       self.bound, stream)
         self._planned = True
 
-    def forward(self, x, stream=None):
-        """route -> histogram -> dispatch -> expert_ffn -> combine on device tensor x [T, D]."""
+    def forward(self, x, stream=None, out=None):
+        """route -> histogram -> dispatch -> expert_ffn -> combine on device tensor x [T, D].
+        The result goes to `out` (bf16 [T, D]) if given, else to the layer's own buffer."""
         if not self._planned:
             raise RuntimeError("call plan(predicted_hist) before forward()")
         c = self.ctx
+        out = self.out if out is None else out
         c.route(x, self.w_router, self.bias, self.topk_idx, self.topk_w, stream)
         c.histogram(self.topk_idx, self.hist, stream)
         c.dispatch(x, self.topk_idx, self.hist, self.replicas, self.slot_off, self.slot_row_off,
                    self.row_pair, self.pair_row, self.xp, self.workspace, stream)
         c.expert_ffn(self.xp, self.slot_row_off, self.slot_expert, self.w_gate, self.w_up,
                      self.w_down, self.h_ws, self.yp, stream)
-        c.combine(self.yp, self.pair_row, self.topk_w, self.out, stream)
-        return self.out
+        c.combine(self.yp, self.pair_row, self.topk_w, out, stream)
+        return out
 
     def forward_host(self, x_host, out_host, stream=None):
         """Same, with (pinned) host tensors: copies x in, runs the layer, copies the result out."""
@@ -65,3 +67,52 @@ class MoeLayer:
         out = self.forward(self.x, stream)
         out_host.copy_(out, non_blocking=True)
         return out_host
+
+
+class HostPipeline:
+    """Streams batches that live in pinned host memory through a MoeLayer.
+
+    The host->device copy of batch i+1 and the device->host copy of result i-1 run on their own
+    streams while batch i computes (PCIe is full duplex), with `depth` device buffers for inputs and
+    results; events order every hand-over.  The layer's compute still runs on the current stream.
+    """
+
+    def __init__(self, layer: MoeLayer, depth: int = 2):
+        s = layer.shape
+        dev = layer.w_router.device
+        self.layer, self.depth, self.n = layer, depth, 0
+        bf = dict(dtype=torch.bfloat16, device=dev)
+        self.x_dev = [torch.empty(s.T, s.D, **bf) for _ in range(depth)]
+        self.out_dev = [torch.empty(s.T, s.D, **bf) for _ in range(depth)]
+        self.s_in, self.s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+        ev = lambda: [torch.cuda.Event() for _ in range(depth)]  # noqa: E731
+        self.ev_in, self.ev_comp, self.ev_out = ev(), ev(), ev()
+
+    def submit(self, x_host, out_host):
+        """Queues one batch: x_host -> device -> layer -> out_host.  Returns immediately."""
+        k = self.n % self.depth
+        compute = torch.cuda.current_stream()
+        reuse = self.n >= self.depth
+        with torch.cuda.stream(self.s_in):
+            if reuse:
+                self.s_in.wait_event(self.ev_comp[k])      # the batch that used this input buffer is done
+            else:
+                self.s_in.wait_stream(compute)             # do not start before work already queued
+            self.x_dev[k].copy_(x_host, non_blocking=True)
+            self.ev_in[k].record(self.s_in)
+        compute.wait_event(self.ev_in[k])
+        if reuse:
+            compute.wait_event(self.ev_out[k])             # the result buffer has been read out
+        self.layer.forward(self.x_dev[k], out=self.out_dev[k])
+        self.ev_comp[k].record(compute)
+        with torch.cuda.stream(self.s_out):
+            self.s_out.wait_event(self.ev_comp[k])
+            out_host.copy_(self.out_dev[k], non_blocking=True)
+            self.ev_out[k].record(self.s_out)
+        self.n += 1
+
+    def drain(self):
+        """Makes the current stream wait for every queued copy (call before timing/reading results)."""
+        compute = torch.cuda.current_stream()
+        compute.wait_stream(self.s_in)
+        compute.wait_stream(self.s_out)

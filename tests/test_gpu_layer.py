@@ -78,6 +78,25 @@ def test_layer_host_buffers():
     assert torch.equal(oh, layer.forward(x.to(DEV)).cpu())
 
 
+def test_host_pipeline_overlapped_copies_give_the_same_results():
+    from paper_2506_07366_b200.layer import HostPipeline
+    w = wl.WORKLOADS["tiny"]
+    _, wr, bias, w1, w3, w2 = build_inputs(w, DEV)
+    shape = binding.Shape(w.T, w.D, w.F, w.E, w.K, w.S, w.gate_mode, 128)
+    layer = MoeLayer(shape, wr.to(DEV), bias.to(DEV), w1.to(DEV), w3.to(DEV), w2.to(DEV))
+    layer.plan(torch.ones(w.E, dtype=torch.int32))
+    batches = [wl.activations(w.scaled(number=w.number + 7 * i), "cpu").pin_memory() for i in range(5)]
+    outs = [torch.zeros(w.T, w.D, dtype=torch.bfloat16).pin_memory() for _ in batches]
+    pipe = HostPipeline(layer, depth=2)
+    for xb, ob in zip(batches, outs):
+        pipe.submit(xb, ob)
+    pipe.drain()
+    torch.cuda.synchronize()
+    layer.ctx.check_status()
+    for xb, ob in zip(batches, outs):
+        assert torch.equal(ob, layer.forward(xb.to(DEV)).cpu())
+
+
 class ExpertsOnDemand:
     """w[e] -> host bf16 bits of one expert's matrix, fetched from the device when asked for."""
 
