@@ -183,6 +183,14 @@ MOEGPS_API int moegps_expert_ffn_down(moegps_ctx_t* ctx, const void* h_ws, const
 MOEGPS_API int moegps_combine(moegps_ctx_t* ctx, const void* yp, const int32_t* pair_row, const float* topk_w,
                    void* out, void* stream);
 
+/* Self-test of the library's failure detection (no counterpart in the paper).  Every wait inside the
+ * pipelined kernels (route, expert_ffn) is bounded: when it runs out the kernel records
+ * MOEGPS_ERR_TIMEOUT in the status word, drains and returns instead of hanging.  This call launches
+ * a one-warp kernel that waits on a barrier nobody signals and gives up after `limit_cycles` SM
+ * cycles (1e3 .. 4e9); afterwards moegps_status reports MOEGPS_ERR_TIMEOUT and the context and the
+ * device are as usable as before. */
+MOEGPS_API int moegps_selftest_bounded_wait(moegps_ctx_t* ctx, int64_t limit_cycles, void* stream);
+
 /* Synchronises `stream`, copies the device status word to *host_status (0 = no device-side error,
  * else the first moegps_error recorded) and clears it.  Returns MOEGPS_OK or MOEGPS_ERR_CUDA. */
 MOEGPS_API int moegps_status(moegps_ctx_t* ctx, void* stream, int32_t* host_status);

@@ -56,6 +56,7 @@ EXPORTS = (
     "moegps_route_logits", "moegps_histogram", "moegps_plan", "moegps_dispatch", "moegps_dispatch_static",
     "moegps_expert_ffn", "moegps_expert_ffn_gate_up", "moegps_expert_ffn_down", "moegps_combine",
     "moegps_status", "moegps_launch_count", "moegps_last_cuda_error", "moegps_error_string",
+    "moegps_selftest_bounded_wait",
 )
 
 
@@ -102,6 +103,7 @@ def _lib():
         "moegps_expert_ffn_gate_up": (ctypes.c_int, [vp] * 8),
         "moegps_expert_ffn_down": (ctypes.c_int, [vp] * 7),
         "moegps_combine": (ctypes.c_int, [vp] * 6),
+        "moegps_selftest_bounded_wait": (ctypes.c_int, [vp, i64, vp]),
         "moegps_status": (ctypes.c_int, [vp, vp, _c_int32_p]),
         "moegps_launch_count": (i64, [vp]),
         "moegps_last_cuda_error": (ctypes.c_int, [vp]),
@@ -276,6 +278,11 @@ class Context:
             _ptr(pair_row, torch.int32, (s.T, s.K), "pair_row"),
             _ptr(topk_w, torch.float32, (s.T, s.K), "topk_w"),
             _ptr(out, torch.bfloat16, (s.T, s.D), "out"), _stream(stream)), "moegps_combine")
+
+    def selftest_bounded_wait(self, limit_cycles: int = 2_000_000, stream=None):
+        """Launches a kernel whose wait can never be satisfied; status() then reports ERR_TIMEOUT."""
+        self._check(_lib().moegps_selftest_bounded_wait(self._h, int(limit_cycles), _stream(stream)),
+                    "moegps_selftest_bounded_wait")
 
     # -- bookkeeping --------------------------------------------------------------------------
     def status(self, stream=None) -> int:

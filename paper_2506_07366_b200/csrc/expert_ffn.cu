@@ -4,7 +4,7 @@
 //   GEMM 2:  Yp = H W2[e]^T
 // Tile = 128 rows of one slot x 256 accumulator columns (GEMM 1: 128 gate + 128 up columns).
 // Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (one elected thread; owns TMEM),
-// warps 2..5 = epilogue (each reads its quarter of the 128 TMEM lanes).  A 4-stage shared-memory ring
+// warps 2..9 = epilogue (two per quarter of the 128 TMEM lanes, half the columns each).  A 4-stage ring
 // (TMA -> tcgen05.mma) and two TMEM accumulators (mainloop of tile i+1 overlaps the epilogue of tile
 // i) are handed around with mbarriers; every wait is bounded and raises an abort flag on expiry.
 // Tiles are enumerated on the device from slot_row_off (no host round trip): slot-major, then

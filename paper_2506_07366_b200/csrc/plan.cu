@@ -1,6 +1,7 @@
-// plan: Algorithm 1 of the paper in slot form, on one CTA.  Thread e keeps (n_e, r_e) in registers;
-// each of the S-E rounds is a block-wide arg-max of n_e / r_e (exact: 64-bit cross-multiplication)
-// that hands the next free slot to the winner.  Integer only.
+// plan: Algorithm 1 of the paper in slot form, on one CTA.  Warp 0 keeps (n_e, r_e) of all experts
+// in registers (lane l: experts l, l+32, ...); each of the S-E rounds is an arg-max of n_e / r_e
+// (exact: 64-bit cross-multiplication) over the lanes' best candidates by a shuffle butterfly, which
+// hands the next free slot to the winner.  The slot tables then come from a block scan.  Integer only.
 #include "common.cuh"
 
 namespace {

@@ -49,7 +49,7 @@ constexpr long long kWaitLimitCycles = 2000000000ll;
 // (an epilogue warp waiting for a whole main loop) should not burn issue slots and power that the
 // tensor pipe needs; latency-critical waits pass 0.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                          unsigned sleep_ns = 0) {
+                                          unsigned sleep_ns = 0, long long limit_cycles = kWaitLimitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   uint32_t spins = 0;
@@ -58,7 +58,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     if (sleep_ns) __nanosleep(sleep_ns);
     if ((++spins & 63u) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitLimitCycles) {
+      if (clock64() - t0 > limit_cycles) {
         *abort_flag = 1;
         return false;
       }

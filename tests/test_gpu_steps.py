@@ -323,6 +323,24 @@ def test_combine(T, D, K, S, A):
     assert np.abs(got - ref).max() <= 2 ** -8 * np.abs(ref).max()
 
 
+def test_bounded_wait_reports_timeout_and_leaves_the_context_usable():
+    # failure detection without a fault: a wait that nothing will ever satisfy must give up, report
+    # through the status word, and let the kernel return; later calls work as usual
+    shape = binding.Shape(64, 64, 64, 4, 2, 4, 0, 1)
+    ctx = binding.Context(shape)
+    assert ctx.status() == 0
+    ctx.selftest_bounded_wait(limit_cycles=2_000_000)          # about a millisecond
+    assert ctx.status() == binding.ERR_TIMEOUT
+    assert ctx.status() == 0
+    idx = torch.randint(0, 4, (64, 2), dtype=torch.int32, device=DEV)
+    hist = poison_i32(4)
+    ctx.histogram(idx, hist)
+    ctx.check_status()
+    assert int(hist.sum()) == 128
+    with pytest.raises(binding.MoegpsError):
+        ctx.selftest_bounded_wait(limit_cycles=10)              # out of the accepted range
+
+
 def test_invalid_pointers_launch_nothing():
     shape = binding.Shape(64, 64, 64, 4, 2, 4, 0, 1)
     ctx = binding.Context(shape)
