@@ -13,6 +13,7 @@ from .moe_oracle import (  # noqa: F401
     p_hat,
     skewness,
     error_rate,
+    predictor_update,
     plan,
     replica_starts,
     dispatch,

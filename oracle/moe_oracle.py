@@ -23,6 +23,7 @@ import numpy as np
 
 __all__ = [
     "bf16_bits_to_f64", "route_logits", "route", "histogram", "p_hat", "skewness", "error_rate",
+    "predictor_update",
     "plan", "replica_starts", "dispatch", "expert_ffn", "combine", "moe_layer",
 ]
 
@@ -131,6 +132,22 @@ def error_rate(p_est, p_true) -> float:
     b = np.asarray(p_true, dtype=np.float64)
     E = a.size
     return float(np.mean(np.abs(a - b) / (1.0 / E)))
+
+
+def predictor_update(state, hist):
+    """Distribution-Only predictor state over batches (Section 3.2.1: with batched data the
+    estimate of Eq. 1 becomes a moving average): the state holds the per-expert counts of all
+    batches seen, so state / sum(state) is the maximum-likelihood estimate over the pooled tokens.
+    Returns (new_state as Python ints, predicted_hist int32): the prediction handed to the planner
+    is the state itself, divided by the smallest power of two that makes its largest entry fit an
+    int32 (only proportions matter to the plan)."""
+    s = [int(a) + int(b) for a, b in zip(np.asarray(state).reshape(-1), np.asarray(hist).reshape(-1))]
+    if any(int(b) < 0 for b in np.asarray(hist).reshape(-1)):
+        raise ValueError("counts must be >= 0")
+    shift = 0
+    while (max(s) >> shift) > 2 ** 31 - 1:
+        shift += 1
+    return s, np.array([v >> shift for v in s], dtype=np.int32)
 
 
 # --------------------------------------------------------------------------------------------

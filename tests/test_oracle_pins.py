@@ -480,3 +480,28 @@ def test_combine_identity_gather_and_linearity():
     assert small.tolist() == [[1.5, 15.0]]
     sub = oracle.combine(yp, pair_row, w, tokens=[3, 17])
     assert np.array_equal(sub[[3, 17]], oracle.combine(yp, pair_row, w)[[3, 17]])
+
+
+# ------------------------------------------------------------------------------ predictor state
+def test_predictor_state_is_the_pooled_mle_and_a_moving_average():
+    E, K = 7, 2
+    batches = [random_routing(T, K, E, 1.1) for T in (40, 40, 40, 40)]
+    state = [0] * E
+    for b in batches:
+        state, pred = oracle.predictor_update(state, oracle.histogram(b, E))
+    pooled = np.bincount(np.concatenate([b.reshape(-1) for b in batches]), minlength=E)
+    assert state == pooled.tolist() and pred.tolist() == pooled.tolist()
+    # Eq. 1 over the pooled tokens; with equal batch sizes that is the plain average of the per-batch estimates
+    per_batch = np.mean([oracle.p_hat(oracle.histogram(b, E)) for b in batches], axis=0)
+    assert np.allclose(oracle.p_hat(pred), per_batch, rtol=1e-12)
+    assert abs(oracle.p_hat(pred).sum() - 1) < 1e-12
+
+
+def test_predictor_scales_huge_counts_by_a_power_of_two():
+    state, pred = oracle.predictor_update([2 ** 33, 2 ** 31, 3], [0, 0, 1])
+    assert state == [2 ** 33, 2 ** 31, 4]
+    assert pred.tolist() == [2 ** 30, 2 ** 28, 0]          # shifted right by 3: the largest fits 31 bits
+    state, pred = oracle.predictor_update([2 ** 31 - 2, 5], [1, 0])
+    assert pred.tolist() == [2 ** 31 - 1, 5]               # still fits: no scaling
+    with pytest.raises(ValueError):
+        oracle.predictor_update([1, 1], [0, -1])
