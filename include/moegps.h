@@ -183,6 +183,23 @@ MOEGPS_API int moegps_expert_ffn_down(moegps_ctx_t* ctx, const void* h_ws, const
 MOEGPS_API int moegps_combine(moegps_ctx_t* ctx, const void* yp, const int32_t* pair_row, const float* topk_w,
                    void* out, void* stream);
 
+/* predictor_update - state of Distribution-Only Prediction across batches (paper, Section 3.2.1:
+ * the maximum-likelihood estimate p_e = n_e / N of Eq. 1, which becomes a moving average when the
+ * data arrive as batches).  state[e] += hist[e]; state / sum(state) is then Eq. 1 over all tokens
+ * seen.  predicted_hist = state divided by the smallest power of two that makes its largest entry fit
+ * an int32 (the planner only uses proportions) - ready to be passed to moegps_plan for the next
+ * batch.  hist: int32 [E] >= 0; state: int64 [E], zeroed by the caller to start or restart;
+ * predicted_hist: int32 [E].  All device pointers, 16-byte aligned. */
+MOEGPS_API int moegps_predictor_update(moegps_ctx_t* ctx, const int32_t* hist, int64_t* state,
+                                       int32_t* predicted_hist, void* stream);
+
+/* error_rate - the paper's quality metric of a predicted distribution (Section 3.2.1, with the
+ * averaging of Section 3.3): mean over the experts of |p_est_e - p_e| / (1/E), where p_est and p are
+ * predicted_hist and hist normalised to sum 1.  fp64, deterministic summation order.
+ * error_rate: double [1] on the device (8-byte aligned); 0 if either histogram is empty. */
+MOEGPS_API int moegps_error_rate(moegps_ctx_t* ctx, const int32_t* predicted_hist, const int32_t* hist,
+                                 double* error_rate, void* stream);
+
 /* Self-test of the library's failure detection (no counterpart in the paper).  Every wait inside the
  * pipelined kernels (route, expert_ffn) is bounded: when it runs out the kernel records
  * MOEGPS_ERR_TIMEOUT in the status word, drains and returns instead of hanging.  This call launches

@@ -56,7 +56,7 @@ EXPORTS = (
     "moegps_route_logits", "moegps_histogram", "moegps_plan", "moegps_dispatch", "moegps_dispatch_static",
     "moegps_expert_ffn", "moegps_expert_ffn_gate_up", "moegps_expert_ffn_down", "moegps_combine",
     "moegps_status", "moegps_launch_count", "moegps_last_cuda_error", "moegps_error_string",
-    "moegps_selftest_bounded_wait",
+    "moegps_selftest_bounded_wait", "moegps_predictor_update", "moegps_error_rate",
 )
 
 
@@ -104,6 +104,8 @@ def _lib():
         "moegps_expert_ffn_down": (ctypes.c_int, [vp] * 7),
         "moegps_combine": (ctypes.c_int, [vp] * 6),
         "moegps_selftest_bounded_wait": (ctypes.c_int, [vp, i64, vp]),
+        "moegps_predictor_update": (ctypes.c_int, [vp] * 5),
+        "moegps_error_rate": (ctypes.c_int, [vp] * 5),
         "moegps_status": (ctypes.c_int, [vp, vp, _c_int32_p]),
         "moegps_launch_count": (i64, [vp]),
         "moegps_last_cuda_error": (ctypes.c_int, [vp]),
@@ -278,6 +280,20 @@ class Context:
             _ptr(pair_row, torch.int32, (s.T, s.K), "pair_row"),
             _ptr(topk_w, torch.float32, (s.T, s.K), "topk_w"),
             _ptr(out, torch.bfloat16, (s.T, s.D), "out"), _stream(stream)), "moegps_combine")
+
+    def predictor_update(self, hist, state, predicted_hist, stream=None):
+        s = self.shape
+        self._check(_lib().moegps_predictor_update(
+            self._h, _ptr(hist, torch.int32, (s.E,), "hist"), _ptr(state, torch.int64, (s.E,), "state"),
+            _ptr(predicted_hist, torch.int32, (s.E,), "predicted_hist"), _stream(stream)),
+            "moegps_predictor_update")
+
+    def error_rate(self, predicted_hist, hist, error_rate, stream=None):
+        s = self.shape
+        self._check(_lib().moegps_error_rate(
+            self._h, _ptr(predicted_hist, torch.int32, (s.E,), "predicted_hist"),
+            _ptr(hist, torch.int32, (s.E,), "hist"), _ptr(error_rate, torch.float64, (1,), "error_rate"),
+            _stream(stream)), "moegps_error_rate")
 
     def selftest_bounded_wait(self, limit_cycles: int = 2_000_000, stream=None):
         """Launches a kernel whose wait can never be satisfied; status() then reports ERR_TIMEOUT."""

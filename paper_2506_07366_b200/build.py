@@ -11,7 +11,7 @@ ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libmoegps.so")
 SOURCES = ["api.cu", "route.cu", "histogram.cu", "plan.cu", "dispatch.cu", "expert_ffn.cu", "combine.cu",
-           "selftest.cu"]
+           "predictor.cu", "selftest.cu"]
 HEADERS = ["common.cuh", "sm100.cuh", "route_epilogue.cuh"]
 
 
