@@ -46,29 +46,32 @@ __device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
   return v;
 }
 
-// One warp per token row: fetch the KS partial logits of the row (own and peers' shared memory),
-// sum them in slice order, add the bias, keep the row in registers (lane l holds experts l,
-// l+32, ...) and select.
-template <int NPL, int KS>
+// One group of G lanes per token row (32/G tokens per warp at a time): fetch the KS partial logits
+// of the row (own and peers' shared memory), sum them in slice order, add the bias, keep the row in
+// registers (sub-lane l holds experts l, l+G, ...) and select.
+template <int NPL, int KS, int G>
 __device__ __forceinline__ void reduce_select(const RouteParams& p, const float* partial, uint32_t rank, int m0,
                                               const float* __restrict__ bias, int32_t* __restrict__ topk_idx,
                                               float* __restrict__ topk_w, float* __restrict__ logits_out) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr int rows_per = BM / KS;
+  constexpr int kTokensPerWarp = 32 / G;
+  const int sl = lane & (G - 1), grp = lane / G;
   uint32_t peer[KS];
 #pragma unroll
   for (int k = 0; k < KS; ++k) peer[k] = map_to_cta(smem_u32(partial), (uint32_t)k);
   float b[NPL];
 #pragma unroll
-  for (int i = 0; i < NPL; ++i) b[i] = (bias && lane + 32 * i < p.E) ? bias[lane + 32 * i] : 0.f;
-  for (int r = warp; r < rows_per; r += kThreads / 32) {
+  for (int i = 0; i < NPL; ++i) b[i] = (bias && sl + G * i < p.E) ? bias[sl + G * i] : 0.f;
+  for (int r0 = warp * kTokensPerWarp; r0 < rows_per; r0 += (kThreads / 32) * kTokensPerWarp) {
+    const int r = r0 + grp;
     const int row = (int)rank * rows_per + r;
     const int t = m0 + row;
-    if (t >= p.T) continue;                              // warp-uniform
+    if (r >= rows_per || t >= p.T) continue;             // uniform within a group
     float raw[NPL][KS];
 #pragma unroll
     for (int i = 0; i < NPL; ++i) {
-      const int e = lane + 32 * i;
+      const int e = sl + G * i;
       const uint32_t off = (uint32_t)((row * p.part_stride + (e < p.E ? e : 0)) * 4);
 #pragma unroll
       for (int k = 0; k < KS; ++k) raw[i][k] = ld_cluster_f32(peer[k] + off);
@@ -84,10 +87,10 @@ __device__ __forceinline__ void reduce_select(const RouteParams& p, const float*
     if (logits_out) {
 #pragma unroll
       for (int i = 0; i < NPL; ++i)
-        if (lane + 32 * i < p.E) logits_out[(int64_t)t * p.E + lane + 32 * i] = v[i];
+        if (sl + G * i < p.E) logits_out[(int64_t)t * p.E + sl + G * i] = v[i];
     }
     if (topk_idx)
-      warp_topk_gate<NPL>(v, p.E, p.K, p.gate_mode, topk_idx + (int64_t)t * p.K, topk_w + (int64_t)t * p.K);
+      group_topk_gate<NPL, G>(v, p.E, p.K, p.gate_mode, topk_idx + (int64_t)t * p.K, topk_w + (int64_t)t * p.K);
   }
 }
 
@@ -201,17 +204,19 @@ route_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
   cluster_sync_all();           // every CTA's partial is complete and visible cluster-wide
 
   // reduction + selection: CTA `rank` owns rows [rank*rows_per, (rank+1)*rows_per) of the tile
-#define MOEGPS_ROUTE_SELECT(NPL)                                                                          \
+#define MOEGPS_ROUTE_SELECT(NPL, G)                                                                       \
   switch (p.ks) {                                                                                         \
-    case 1: reduce_select<NPL, 1>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out); break;       \
-    case 2: reduce_select<NPL, 2>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out); break;       \
-    case 4: reduce_select<NPL, 4>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out); break;       \
-    default: reduce_select<NPL, 8>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out); break;      \
+    case 1: reduce_select<NPL, 1, G>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out); break;    \
+    case 2: reduce_select<NPL, 2, G>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out); break;    \
+    case 4: reduce_select<NPL, 4, G>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out); break;    \
+    default: reduce_select<NPL, 8, G>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out); break;   \
   }
-  if (p.E <= 32) { MOEGPS_ROUTE_SELECT(1) }
-  else if (p.E <= 64) { MOEGPS_ROUTE_SELECT(2) }
-  else if (p.E <= 128) { MOEGPS_ROUTE_SELECT(4) }
-  else { MOEGPS_ROUTE_SELECT(8) }
+  if (p.E <= 8) { MOEGPS_ROUTE_SELECT(1, 8) }            // four tokens per warp at a time
+  else if (p.E <= 16) { MOEGPS_ROUTE_SELECT(1, 16) }     // two
+  else if (p.E <= 32) { MOEGPS_ROUTE_SELECT(1, 32) }
+  else if (p.E <= 64) { MOEGPS_ROUTE_SELECT(2, 32) }
+  else if (p.E <= 128) { MOEGPS_ROUTE_SELECT(4, 32) }
+  else { MOEGPS_ROUTE_SELECT(8, 32) }
 #undef MOEGPS_ROUTE_SELECT
   __syncwarp();
   cluster_sync_all();           // nobody leaves while a peer may still read its shared memory
@@ -231,7 +236,7 @@ int moegps_launch_route(moegps_ctx* ctx, const void* x, const void* wr, const fl
   p.e_pad = (s.E + 15) / 16 * 16;
   const int stage_bytes = kABytes + p.e_pad * 128;
   p.stages = 196608 / stage_bytes;          // ring of at most 192 KiB
-  if (p.stages > 8) p.stages = 8;
+  if (p.stages > 10) p.stages = 10;
   const int nkb = (s.D + BK - 1) / BK;
   const int tiles = (s.T + BM - 1) / BM;
   // split the model dimension until the grid covers most of the chip (cluster size <= 8, a power
