@@ -81,3 +81,14 @@ def test_context_needs_a_gpu(lib):
         pytest.skip("a GPU is present")
     with pytest.raises(RuntimeError):
         binding.Context(binding.Shape(T=8, D=64, F=64, E=2, K=1, S=2))
+
+
+def test_missing_library_fails_loudly(tmp_path):
+    # there is no fallback path: a missing shared library must raise, in a fresh interpreter
+    import subprocess
+    import sys
+    code = ("import os, sys; sys.path.insert(0, %r); os.environ['MOEGPS_LIBRARY'] = %r; "
+            "from paper_2506_07366_b200 import binding; binding._lib()") % (ROOT, str(tmp_path / "nope.so"))
+    proc = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True)
+    assert proc.returncode != 0
+    assert "ImportError" in proc.stderr and "no fallback" in proc.stderr
