@@ -40,7 +40,9 @@ struct __align__(16) Tables {
   int32_t expert[kMaxS];
 };
 
-constexpr size_t kSmemBytes = 1024 /* alignment slack */ + (size_t)kStages * kStageBytes + sizeof(Tables) + 256;
+constexpr int kEpilogueWarps = 8;
+constexpr size_t kSmemBytes = 1024 /* alignment slack */ + (size_t)kStages * kStageBytes + sizeof(Tables) + 256 +
+                              kEpilogueWarps * 32 * 80 /* epilogue staging */;
 
 struct TileCoord {
   int m0;        // first row of the tile in the permuted buffer
@@ -83,52 +85,57 @@ __device__ __forceinline__ float silu_fast(float g) {
   return g * fmaf(0.5f, t, 0.5f);
 }
 
-// Epilogue of one tile for one thread (= one accumulator row): TMEM -> registers -> bf16 -> global.
+// Epilogue of one tile for one warp: 32 accumulator rows (one per lane) x half of the tile's output
+// columns, TMEM -> registers -> bf16 -> shared-memory staging -> global.
 // kSwiGLU: columns [0,128) are the gate and [128,256) the up projection; 128 outputs silu(g)*u.
-// `half` (0 or 1) selects which half of the tile's output columns this warp drains: two warps share
-// each quarter of the TMEM lanes.
+// `half` (0 or 1) selects which half of the output columns this warp drains (two warps share each
+// quarter of the TMEM lanes).  A lane owns one row, so storing straight from registers would
+// scatter 16-byte pieces over 32 rows per instruction - measured to cost the main loop 5-14 % of its
+// L2/HBM throughput.  Instead each 32-column chunk (64 bytes per row) goes through a per-warp
+// staging buffer (rows 80 bytes apart: conflict-free) and is written out with four lanes per row,
+// i.e. whole 64-byte segments.  `row0` is the first of the warp's 32 rows, `row_end` the slot's end.
+constexpr int kStageRowBytes = 80;
+constexpr int kStagingBytesPerWarp = 32 * kStageRowBytes;
+
 template <bool kSwiGLU>
-__device__ __forceinline__ void drain_tile(uint32_t taddr, bool row_ok, __nv_bfloat16* orow, int col0, int n_dim,
-                                           int half) {
-if constexpr (kSwiGLU) {
+__device__ __forceinline__ void drain_tile(uint32_t taddr, uint8_t* staging, int lane, __nv_bfloat16* out,
+                                           int row0, int row_end, int col0, int n_dim, int half) {
+  constexpr int kCols = kSwiGLU ? 128 : 256;          // output columns of a tile
 #pragma unroll 1
-  for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 32) {
-    uint32_t g[32], u[32];
-    tmem_ld32(taddr + c0, g);
-    tmem_ld32(taddr + 128 + c0, u);
-    tmem_ld_wait();
+  for (int c0 = (kCols / 2) * half; c0 < (kCols / 2) * (half + 1); c0 += 32) {
     uint32_t o[16];
+    if constexpr (kSwiGLU) {
+      uint32_t g[32], u[32];
+      tmem_ld32(taddr + c0, g);
+      tmem_ld32(taddr + 128 + c0, u);
+      tmem_ld_wait();
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
-      const float h0 = silu_fast(g0) * __uint_as_float(u[2 * i]);
-      const float h1 = silu_fast(g1) * __uint_as_float(u[2 * i + 1]);
-      o[i] = pack_bf16(h0, h1);
-    }
-    if (row_ok) {
+      for (int i = 0; i < 16; ++i) {
+        const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
+        o[i] = pack_bf16(silu_fast(g0) * __uint_as_float(u[2 * i]), silu_fast(g1) * __uint_as_float(u[2 * i + 1]));
+      }
+    } else {
+      uint32_t a[32];
+      tmem_ld32(taddr + c0, a);
+      tmem_ld_wait();
 #pragma unroll
-      for (int v = 0; v < 4; ++v)
-        if (col0 + c0 + 8 * v + 8 <= n_dim)
-          *reinterpret_cast<uint4*>(orow + c0 + 8 * v) = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
+      for (int i = 0; i < 16; ++i) o[i] = pack_bf16(__uint_as_float(a[2 * i]), __uint_as_float(a[2 * i + 1]));
     }
+    uint4* mine = reinterpret_cast<uint4*>(staging + lane * kStageRowBytes);
+#pragma unroll
+    for (int v = 0; v < 4; ++v) mine[v] = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
+    __syncwarp();
+    const int piece = lane & 3;                       // which 16 bytes of the row's 64
+    const int col = col0 + c0 + 8 * piece;
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+      const int r = it * 8 + (lane >> 2);
+      const uint4 val = *reinterpret_cast<const uint4*>(staging + r * kStageRowBytes + piece * 16);
+      const int row = row0 + r;
+      if (row < row_end && col + 8 <= n_dim) *reinterpret_cast<uint4*>(out + (size_t)row * n_dim + col) = val;
+    }
+    __syncwarp();
   }
-} else {
-#pragma unroll 1
-  for (int c0 = 128 * half; c0 < 128 * half + 128; c0 += 32) {
-    uint32_t a[32];
-    tmem_ld32(taddr + c0, a);
-    tmem_ld_wait();
-    uint32_t o[16];
-#pragma unroll
-    for (int i = 0; i < 16; ++i) o[i] = pack_bf16(__uint_as_float(a[2 * i]), __uint_as_float(a[2 * i + 1]));
-    if (row_ok) {
-#pragma unroll
-      for (int v = 0; v < 4; ++v)
-        if (col0 + c0 + 8 * v + 8 <= n_dim)
-          *reinterpret_cast<uint4*>(orow + c0 + 8 * v) = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
-    }
-  }
-}
 }
 
 // kSwiGLU = true : out[row, n_tile*128 + c] = silu(acc[c]) * acc[128 + c],  c < 128
@@ -252,7 +259,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
   } else {
     const int quarter = warp & 3;                 // TMEM lanes this warp may read
     const int half = (warp - 2) >> 2;             // which half of the output columns it drains
-    const int row_in_tile = quarter * 32 + lane;
+    uint8_t* staging = smem + (size_t)kStages * kStageBytes + sizeof(Tables) + 256 + (warp - 2) * kStagingBytesPerWarp;
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
@@ -261,11 +268,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
       if (!mbar_wait(&acc_full[acc], acc_phase, abort_flag, 256)) { ok = false; break; }
       tc_fence_after_sync();
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * BNACC;
-      const int row = tc.m0 + row_in_tile;
-      const bool row_ok = row < tc.row_end;
       const int col0 = tc.n_tile * cols_per_tile;
-      __nv_bfloat16* orow = out + (size_t)row * n_dim + col0;
-      drain_tile<kSwiGLU>(taddr, row_ok, orow, col0, n_dim, half);
+      drain_tile<kSwiGLU>(taddr, staging, lane, out, tc.m0 + quarter * 32, tc.row_end, col0, n_dim, half);
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(&acc_empty[acc]);
