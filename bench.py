@@ -263,6 +263,14 @@ def run_ours(args):
     achieved = flops_gate_up / (gate_up_ms * 1e-3) / 1e12
     ffn_tflops = 6.0 * w.R * w.D * w.F / ((gate_up_ms + down_ms) * 1e-3) / 1e12
     hist_np = true_hist.numpy().astype("float64")
+    # slot loads of the last step: rows that carry a pair, counted per slot
+    occupied = (layer.row_pair >= 0).to(torch.int64).cumsum(0)
+    ends = layer.slot_row_off[1:].long().clamp(max=shape.Rcap) - 1
+    starts = layer.slot_row_off[:-1].long() - 1
+    cum_at = lambda i: torch.where(i >= 0, occupied[i.clamp(min=0)], torch.zeros_like(i))  # noqa: E731
+    slot_loads = (cum_at(ends) - cum_at(starts)).cpu().numpy()
+    err_dev = torch.zeros(1, dtype=torch.float64, device=dev)
+    ctx.error_rate(pred_dev, layer.hist, err_dev)
     # a timed region of a few hundred ms runs at boost clocks: the burst peak is the fair denominator;
     # from a couple of seconds on, the power cap has settled and the sustained peak applies
     if elapsed_ms >= 2000.0:
@@ -276,6 +284,12 @@ def run_ours(args):
         "config": {"workload": w.name, "T": w.T, "D": w.D, "F": w.F, "E": w.E, "K": w.K, "S": w.S,
                    "row_align": A, "tokens_per_gpu": w.T, "prediction": w.prediction,
                    "skewness": float(hist_np.max() / (hist_np.sum() / w.E)),
+                   # the paper's load statistics of this batch, from the library's own outputs: the
+                   # bottleneck slot's load over the even share after duplication, the planner's
+                   # predicted bound, and the error rate of the prediction that drove the plan
+                   "skewness_after_plan": float(slot_loads.max() / (w.R / w.S)),
+                   "max_slot_load": int(slot_loads.max()), "plan_bound": int(layer.bound.item()),
+                   "prediction_error_rate": float(err_dev.item()),
                    "l2": "inputs larger than L2: %.2f GB of expert weights stream through it every step"
                          % (3 * w.E * w.D * w.F * 2 / 1e9)},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": w.T * w.D * 2,
