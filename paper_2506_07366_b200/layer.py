@@ -61,6 +61,36 @@ class MoeLayer:
         c.combine(self.yp, self.pair_row, self.topk_w, out, stream)
         return out
 
+    def capture(self, x, predicted_hist=None):
+        """Records plan (if `predicted_hist`, an int32 [E] device tensor, is given) + forward on the
+        fixed tensors `x` / `predicted_hist` into a CUDA graph and returns it; `graph.replay()` then
+        runs the whole step with one launch, reading whatever those tensors hold at that moment and
+        writing `self.out`.  Worth it for small, launch-bound batches (the 8 kernels of a tiny step
+        take 0.12 ms launched one by one and 0.05 ms replayed).  The library's one-time set-up
+        (tensor-map encoding, shared-memory opt-in) happens in the warm-up calls made here."""
+        if predicted_hist is not None:
+            self.pred.copy_(predicted_hist.to(torch.int32))
+        elif not self._planned:
+            raise RuntimeError("call plan(predicted_hist) first or pass predicted_hist")
+        side = torch.cuda.Stream(x.device)
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+
+        def step():
+            if predicted_hist is not None:
+                self.pred.copy_(predicted_hist, non_blocking=True)
+                self.ctx.plan(self.pred, self.shape.S, self.replicas, self.slot_off, self.slot_expert, self.bound)
+                self._planned = True
+            self.forward(x)
+
+        with torch.cuda.stream(side):
+            for _ in range(2):
+                step()
+            with torch.cuda.graph(graph, stream=side):
+                step()
+        torch.cuda.current_stream().wait_stream(side)
+        return graph
+
     def forward_host(self, x_host, out_host, stream=None):
         """Same, with (pinned) host tensors: copies x in, runs the layer, copies the result out."""
         self.x.copy_(x_host, non_blocking=True)

@@ -97,6 +97,26 @@ def test_host_pipeline_overlapped_copies_give_the_same_results():
         assert torch.equal(ob, layer.forward(xb.to(DEV)).cpu())
 
 
+def test_captured_graph_replays_the_step_on_new_inputs():
+    w = wl.WORKLOADS["tiny"]
+    _, wr, bias, w1, w3, w2 = build_inputs(w, DEV)
+    shape = binding.Shape(w.T, w.D, w.F, w.E, w.K, w.S + 3, w.gate_mode, 128)
+    layer = MoeLayer(shape, wr.to(DEV), bias.to(DEV), w1.to(DEV), w3.to(DEV), w2.to(DEV))
+    x = wl.activations(w, DEV)
+    pred = torch.ones(w.E, dtype=torch.int32, device=DEV)
+    graph = layer.capture(x, pred)
+    for i in range(3):
+        x.copy_(wl.activations(w.scaled(number=w.number + 3 + i), DEV))      # new batch, same buffers
+        pred.copy_(torch.randint(0, 100, (w.E,), dtype=torch.int32, device=DEV))
+        graph.replay()
+        torch.cuda.synchronize()
+        got, got_rep = layer.out.clone(), layer.replicas.clone()
+        layer.plan(pred)
+        want = layer.forward(x).clone()
+        layer.ctx.check_status()
+        assert torch.equal(got, want) and torch.equal(got_rep, layer.replicas)
+
+
 class ExpertsOnDemand:
     """w[e] -> host bf16 bits of one expert's matrix, fetched from the device when asked for."""
 
