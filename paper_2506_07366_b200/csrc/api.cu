@@ -49,6 +49,7 @@ int moegps_create(moegps_ctx_t** out, const moegps_shape_t* shape, int device) {
   ctx->ffn_attr_done = false;
   ctx->rt_valid = false;
   ctx->route_attr_done = false;
+  ctx->dispatch_attr_done = false;
   ctx->d_status = nullptr;
   int prev = 0;
   cudaGetDevice(&prev);

@@ -29,6 +29,7 @@ struct moegps_ctx {
   CUtensorMap tm_rx, tm_rw;
   bool rt_valid;
   bool route_attr_done;
+  bool dispatch_attr_done;
 };
 
 #define MOEGPS_CUDA_TRY(ctx, expr)                                   \

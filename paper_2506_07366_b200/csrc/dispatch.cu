@@ -21,7 +21,7 @@ constexpr int kThreads = kWarpsPerBlock * 32;
 constexpr int kMaxE = 256;
 constexpr int kMaxS = 1024;
 constexpr int kScanThreads = 1024;
-constexpr int kScanSmemBytes = 40 * 1024;   // with the static tables this stays under the 48 KiB default limit
+constexpr int kScanSmemBytes = 100 * 1024;  // staging of the count matrix; two such CTAs still fit one SM
 
 static_assert(kSegPairs == 256, "count_scan assigns one of its first 256 threads to each pair of a segment");
 
@@ -78,10 +78,23 @@ count_scan_kernel(const int32_t* __restrict__ topk_idx, int64_t R, int E, int S,
   for (int e0 = 0; e_chunk > 0 && e0 < E; e0 += e_chunk) {
     const int ec = min(e_chunk, E - e0);
     const int ecp = ec | 1;                     // odd row stride: a column walk hits distinct banks
-    const int n = nseg * ec;
-    for (int i = tid; i < n; i += blockDim.x) {
-      const int g = i / ec, e = i - g * ec;
-      scan_mat[g * ecp + e] = __ldcg(&seg_cnt[(int64_t)g * E + e0 + e]);
+    // thread layout for the copies: tx walks the expert columns (a power of two >= ec lanes wide),
+    // ty the segments - no integer divisions in the loops
+    int tpr_log = 0;
+    while ((1 << tpr_log) < ec && tpr_log < 8) ++tpr_log;
+    const int tx = tid & ((1 << tpr_log) - 1), ty = tid >> tpr_log, rows_per_pass = kScanThreads >> tpr_log;
+    for (int g0 = ty; g0 < nseg; g0 += 4 * rows_per_pass) {   // four independent loads in flight per thread
+      int val[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int g = g0 + u * rows_per_pass;
+        val[u] = (g < nseg && tx < ec) ? __ldcg(&seg_cnt[(int64_t)g * E + e0 + tx]) : 0;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int g = g0 + u * rows_per_pass;
+        if (g < nseg && tx < ec) scan_mat[g * ecp + tx] = val[u];
+      }
     }
     __syncthreads();
     for (int c = warp; c < ec; c += kScanThreads / 32) {      // one warp per expert column
@@ -101,10 +114,8 @@ count_scan_kernel(const int32_t* __restrict__ topk_idx, int64_t R, int E, int S,
       if (lane == 0 && running != hist[e0 + c]) moegps_report(status, MOEGPS_ERR_HIST_MISMATCH, e0 + c);
     }
     __syncthreads();
-    for (int i = tid; i < n; i += blockDim.x) {
-      const int g = i / ec, e = i - g * ec;
-      seg_cnt[(int64_t)g * E + e0 + e] = scan_mat[g * ecp + e];
-    }
+    for (int g = ty; g < nseg; g += rows_per_pass)
+      if (tx < ec) seg_cnt[(int64_t)g * E + e0 + tx] = scan_mat[g * ecp + tx];
     __syncthreads();
   }
   // fallback for pair lists too long for shared memory: a warp per expert, lanes stride the segments
@@ -258,6 +269,11 @@ int moegps_launch_dispatch(moegps_ctx* ctx, const void* x, const int32_t* topk_i
   if (e_chunk > s.E) e_chunk = s.E;
   if (e_chunk < 0) e_chunk = 0;
   const size_t scan_smem = e_chunk > 0 ? (size_t)(e_chunk | 1) * (nseg > 0 ? nseg : 1) * sizeof(int32_t) : 0;
+  if (!ctx->dispatch_attr_done) {
+    MOEGPS_CUDA_TRY(ctx, cudaFuncSetAttribute(count_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              kScanSmemBytes + 1024));
+    ctx->dispatch_attr_done = true;
+  }
   count_scan_kernel<<<nseg > 0 ? nseg : 1, kScanThreads, scan_smem, st>>>(
       topk_idx, R, s.E, s.S, s.row_align, seg, nseg, row_pair, Rcap, hist, replicas, slot_off, slot_row_off, e_chunk,
       ctx->d_status);
