@@ -1,16 +1,22 @@
 // dispatch: the routing shuffle on one device (paper, Section 2; replica choice of Algorithm 1).
 //
 // The flat pair list is cut into segments of kSegPairs consecutive pairs.  Two kernels:
-//   1. count_scan : one CTA per segment counts its pairs per expert (warp match + shared counters)
-//                   into workspace[seg][e] and fills row_pair with -1; the CTA that finishes last
-//                   (ticket counter, no waiting) turns the counts into per-expert exclusive prefix
-//                   sums over the segments and derives the slot row offsets from hist / replicas /
-//                   row_align with a block scan
+//   1. count      : one CTA per segment counts its pairs per expert (warp match + shared counters)
+//                   into the workspace and fills row_pair with -1.
+//                   Up to kDirectMaxSeg segments (262144 pairs): the counts are stored expert-major,
+//                   workspace[e][seg], and CTA 0 also derives the slot row offsets from hist /
+//                   replicas / row_align (they do not depend on the counts) with a block scan.
+//                   Longer pair lists (count_scan): counts are stored workspace[seg][e] and the CTA
+//                   that finishes last (ticket counter, no waiting) turns them into per-expert
+//                   exclusive prefix sums over the segments before it derives the offsets.
 //   2. rank_copy  : one warp per token.  The stable rank of a pair is its segment's base plus the
 //                   number of earlier same-expert pairs inside the segment, which the warp counts
-//                   from the segment's indices (a 1 KiB read); replica, slot and row follow in
-//                   integer arithmetic.  The warp then reads the token row once (128-bit loads) and
-//                   writes it to its K rows of the permuted buffer (128-bit stores).
+//                   from the segment's indices (a 1 KiB read).  The base is read from the scanned
+//                   matrix, or (short lists) summed by the warp from the expert's row of counts -
+//                   a coalesced read of at most 4 KiB that replaces the serial scan, which was a
+//                   chain of dependent global round trips on one SM.  Replica, slot and row follow
+//                   in integer arithmetic.  The warp then reads the token row once (128-bit loads)
+//                   and writes it to its K rows of the permuted buffer (128-bit stores).
 // Stable by construction, integer only, no atomics on results => bit-exact and deterministic.
 #include "common.cuh"
 
@@ -23,7 +29,100 @@ constexpr int kMaxS = 1024;
 constexpr int kScanThreads = 1024;
 constexpr int kScanSmemBytes = 100 * 1024;  // staging of the count matrix; two such CTAs still fit one SM
 
-static_assert(kSegPairs == 256, "count_scan assigns one of its first 256 threads to each pair of a segment");
+static_assert(kSegPairs == 256, "the count kernels assign one thread to each pair of a segment");
+static_assert(kMaxS <= 4 * kSegPairs, "count_kernel scans four slots per thread");
+
+constexpr int kDirectMaxSeg = 1024;   // up to this many segments rank_copy sums the counts itself
+
+// Rows reserved for the replicas of expert `e` (loads rounded up to A) -> padded[slot].
+// Replica rho takes ranks floor(rho n/r) .. floor((rho+1) n/r) - 1.
+__device__ __forceinline__ void slot_loads_of_expert(int e, int S, int A, const int32_t* __restrict__ hist,
+                                                     const int32_t* __restrict__ replicas,
+                                                     const int32_t* __restrict__ slot_off, int32_t* padded,
+                                                     int32_t* status) {
+  const long long n = hist[e];
+  const int r = replicas[e];
+  const int so = slot_off[e];
+  if (r < 1 || so < 0 || so + r > S || n < 0) {
+    moegps_report(status, MOEGPS_ERR_BAD_INDEX, e);
+    return;
+  }
+  // floor(rho n / r) = rho q + floor(rho m / r) with n = q r + m: one division, then 32-bit work
+  const int q = (int)(n / r), m = (int)(n - (long long)q * r);
+  int prev = 0;
+  for (int rho = 1; rho <= r; ++rho) {
+    const int start = rho * q + (rho * m) / r;     // rho, m < r <= 1024
+    padded[so + rho - 1] = (start - prev + A - 1) / A * A;
+    prev = start;
+  }
+}
+
+// Short pair lists: counts only, stored expert-major; CTA 0 also builds slot_row_off.
+__global__ void __launch_bounds__(kSegPairs)
+count_kernel(const int32_t* __restrict__ topk_idx, int64_t R, int E, int S, int A, int32_t* __restrict__ cnt_t,
+             int nseg, int32_t* __restrict__ row_pair, int64_t Rcap, const int32_t* __restrict__ hist,
+             const int32_t* __restrict__ replicas, const int32_t* __restrict__ slot_off,
+             int32_t* __restrict__ slot_row_off, int32_t* status) {
+  __shared__ int32_t cnt[kMaxE];
+  __shared__ int32_t padded[kMaxS];
+  __shared__ int32_t warp_tot[kSegPairs / 32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int seg = blockIdx.x;
+  // padding rows keep -1: fill everything, occupied rows are overwritten by rank_copy
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + tid; i < Rcap; i += (int64_t)gridDim.x * blockDim.x)
+    row_pair[i] = -1;
+  for (int e = tid; e < E; e += kSegPairs) cnt[e] = 0;
+  __syncthreads();
+  {
+    const int64_t p = (int64_t)seg * kSegPairs + tid;
+    int e = -1;
+    if (p < R) {
+      e = topk_idx[p];
+      if (e < 0 || e >= E) {
+        moegps_report(status, MOEGPS_ERR_BAD_INDEX, (int)(p & 0x7fffffff));
+        e = -1;
+      }
+    }
+    const unsigned same = __match_any_sync(0xffffffffu, e);
+    if (e >= 0 && lane == (31 - __clz(same))) atomicAdd(&cnt[e], __popc(same));   // one add per warp and expert
+  }
+  __syncthreads();
+  if (seg < nseg)
+    for (int e = tid; e < E; e += kSegPairs) cnt_t[(int64_t)e * nseg + seg] = cnt[e];
+  if (blockIdx.x != 0) return;
+
+  // ---- CTA 0: slot row offsets (independent of the counts) ----
+  for (int s = tid; s < S; s += kSegPairs) padded[s] = 0;
+  __syncthreads();
+  for (int e = tid; e < E; e += kSegPairs) slot_loads_of_expert(e, S, A, hist, replicas, slot_off, padded, status);
+  __syncthreads();
+  // slot starts are multiples of A, so the offsets are a plain prefix sum of the padded loads;
+  // thread t owns slots 4t .. 4t+3 (S <= 1024 = 4 * 256)
+  int v[4], sum = 0;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int s = 4 * tid + i;
+    v[i] = s < S ? padded[s] : 0;
+    sum += v[i];
+  }
+  int incl = sum;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const int o = __shfl_up_sync(0xffffffffu, incl, d);
+    if (lane >= d) incl += o;
+  }
+  if (lane == 31) warp_tot[warp] = incl;
+  __syncthreads();
+  int run = incl - sum;
+  for (int wv = 0; wv < warp; ++wv) run += warp_tot[wv];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int s = 4 * tid + i;
+    run += v[i];
+    if (s < S) slot_row_off[s + 1] = run;
+  }
+  if (tid == 0) slot_row_off[0] = 0;
+}
 
 __global__ void __launch_bounds__(kScanThreads)
 count_scan_kernel(const int32_t* __restrict__ topk_idx, int64_t R, int E, int S, int A,
@@ -135,24 +234,8 @@ count_scan_kernel(const int32_t* __restrict__ topk_idx, int64_t R, int E, int S,
     }
     if (lane == 0 && running != hist[e]) moegps_report(status, MOEGPS_ERR_HIST_MISMATCH, e);
   }
-  // (b) slot loads: replica rho of expert e takes ranks floor(rho n/r) .. floor((rho+1) n/r) - 1
-  if (tid < E) {
-    const long long n = hist[tid];
-    const int r = replicas[tid];
-    const int so = slot_off[tid];
-    if (r < 1 || so < 0 || so + r > S || n < 0) {
-      moegps_report(status, MOEGPS_ERR_BAD_INDEX, tid);
-    } else {
-      // floor(rho n / r) = rho q + floor(rho m / r) with n = q r + m: one division, then 32-bit work
-      const int q = (int)(n / r), m = (int)(n - (long long)q * r);
-      int prev = 0;
-      for (int rho = 1; rho <= r; ++rho) {
-        const int start = rho * q + (rho * m) / r;     // rho, m < r <= 1024
-        padded[so + rho - 1] = (start - prev + A - 1) / A * A;
-        prev = start;
-      }
-    }
-  }
+  // (b) slot loads
+  if (tid < E) slot_loads_of_expert(tid, S, A, hist, replicas, slot_off, padded, status);
   __syncthreads();
   // slot starts are multiples of A, so the offsets are a plain prefix sum of the padded loads
   const int v = tid < S ? padded[tid] : 0;
@@ -170,40 +253,69 @@ count_scan_kernel(const int32_t* __restrict__ topk_idx, int64_t R, int E, int S,
   if (tid == 0) slot_row_off[0] = 0;
 }
 
+// kDirect: `seg_base` holds the raw counts expert-major ([E][nseg]) and the warp sums the expert's
+// row up to its segment itself; otherwise it holds the scanned matrix ([nseg][E]).
+template <bool kDirect>
 __global__ void __launch_bounds__(kThreads)
 rank_copy_kernel(const uint4* __restrict__ x, int T, int K, int chunks /* D*2/16 */,
                  const int32_t* __restrict__ topk_idx, int64_t R, int E, int S, int64_t Rcap,
-                 const int32_t* __restrict__ seg_base, const int32_t* __restrict__ hist,
+                 const int32_t* __restrict__ seg_base, int nseg, const int32_t* __restrict__ hist,
                  const int32_t* __restrict__ replicas, const int32_t* __restrict__ slot_off,
                  const int32_t* __restrict__ slot_row_off, int32_t* __restrict__ pair_row,
                  int32_t* __restrict__ row_pair, uint4* __restrict__ xp, int32_t* __restrict__ status) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (kDirect && blockIdx.x == 0) {
+    // the counts must add up to the histogram the caller passed (the scan path checks the same)
+    for (int e = warp; e < E; e += kWarpsPerBlock) {
+      int tot = 0;
+      for (int g = lane; g < nseg; g += 32) tot += seg_base[(int64_t)e * nseg + g];
+      tot = __reduce_add_sync(0xffffffffu, tot);
+      if (lane == 0 && tot != hist[e]) moegps_report(status, MOEGPS_ERR_HIST_MISMATCH, e);
+    }
+  }
   const int t = blockIdx.x * kWarpsPerBlock + warp;
   if (t >= T) return;
   // ---- ranks of this token's K pairs ----
-  int my_rank = -1, my_e = -1;                 // lane j < K ends up holding pair j
+  int my_rank = -1, my_e = -1, my_base = 0;    // lane j < K ends up holding pair j
   int64_t cur_seg = -1;
   int v[kSegPairs / 32];
-  for (int j = 0; j < K; ++j) {
-    const int64_t p = (int64_t)t * K + j;
-    const int64_t seg = p / kSegPairs;
-    if (seg != cur_seg) {                      // (re)load the segment's indices, 8 per lane
-      cur_seg = seg;
+  int part[8];                                 // this lane's share of the rank of pair j
 #pragma unroll
-      for (int i = 0; i < kSegPairs / 32; ++i) {
-        const int64_t q = seg * kSegPairs + lane + 32 * i;
-        v[i] = q < R ? topk_idx[q] : -1;
+  for (int j = 0; j < 8; ++j) {
+    part[j] = 0;
+    if (j < K) {
+      const int64_t p = (int64_t)t * K + j;
+      const int64_t seg = p / kSegPairs;
+      if (seg != cur_seg) {                    // (re)load the segment's indices, 8 per lane
+        cur_seg = seg;
+#pragma unroll
+        for (int i = 0; i < kSegPairs / 32; ++i) {
+          const int64_t q = seg * kSegPairs + lane + 32 * i;
+          v[i] = q < R ? topk_idx[q] : -1;
+        }
+      }
+      const int e = topk_idx[p];
+      const int p_local = (int)(p - seg * kSegPairs);
+      int c = 0;
+#pragma unroll
+      for (int i = 0; i < kSegPairs / 32; ++i) c += (lane + 32 * i < p_local && v[i] == e) ? 1 : 0;
+      const bool valid = e >= 0 && e < E;
+      if (kDirect && valid) {
+        const int32_t* row = seg_base + (int64_t)e * nseg;
+        for (int g = lane; g < (int)seg; g += 32) c += row[g];
+      }
+      part[j] = c;
+      if (lane == j) {
+        my_e = e;
+        if (!kDirect && valid) my_base = seg_base[seg * E + e];
       }
     }
-    const int e = topk_idx[p];
-    const int p_local = (int)(p - seg * kSegPairs);
-    int c = 0;
+  }
 #pragma unroll
-    for (int i = 0; i < kSegPairs / 32; ++i) c += (lane + 32 * i < p_local && v[i] == e) ? 1 : 0;
-    c = __reduce_add_sync(0xffffffffu, c);
-    if (lane == j) {
-      my_e = e;
-      my_rank = (e >= 0 && e < E) ? seg_base[seg * E + e] + c : -1;
+  for (int j = 0; j < 8; ++j) {
+    if (j < K) {
+      const int rank = __reduce_add_sync(0xffffffffu, part[j]);
+      if (lane == j) my_rank = (my_e >= 0 && my_e < E) ? my_base + rank : -1;
     }
   }
   // ---- replica, slot, row (lane j for pair j) ----
@@ -274,15 +386,27 @@ int moegps_launch_dispatch(moegps_ctx* ctx, const void* x, const int32_t* topk_i
                                               kScanSmemBytes + 1024));
     ctx->dispatch_attr_done = true;
   }
-  count_scan_kernel<<<nseg > 0 ? nseg : 1, kScanThreads, scan_smem, st>>>(
-      topk_idx, R, s.E, s.S, s.row_align, seg, nseg, row_pair, Rcap, hist, replicas, slot_off, slot_row_off, e_chunk,
-      ctx->d_status);
+  const bool direct = nseg <= kDirectMaxSeg;
+  if (direct) {
+    count_kernel<<<nseg > 0 ? nseg : 1, kSegPairs, 0, st>>>(topk_idx, R, s.E, s.S, s.row_align, seg, nseg, row_pair, Rcap,
+                                                            hist, replicas, slot_off, slot_row_off, ctx->d_status);
+  } else {
+    count_scan_kernel<<<nseg, kScanThreads, scan_smem, st>>>(topk_idx, R, s.E, s.S, s.row_align, seg, nseg, row_pair,
+                                                             Rcap, hist, replicas, slot_off, slot_row_off, e_chunk,
+                                                             ctx->d_status);
+  }
   MOEGPS_AFTER_LAUNCH(ctx);
   if (R == 0) return MOEGPS_OK;
   const int tblocks = (s.T + kWarpsPerBlock - 1) / kWarpsPerBlock;
-  rank_copy_kernel<<<tblocks, kThreads, 0, st>>>(static_cast<const uint4*>(x), s.T, s.K, s.D / 8, topk_idx, R, s.E,
-                                                 s.S, Rcap, seg, hist, replicas, slot_off, slot_row_off, pair_row,
-                                                 row_pair, static_cast<uint4*>(xp), ctx->d_status);
+  if (direct) {
+    rank_copy_kernel<true><<<tblocks, kThreads, 0, st>>>(
+        static_cast<const uint4*>(x), s.T, s.K, s.D / 8, topk_idx, R, s.E, s.S, Rcap, seg, nseg, hist, replicas, slot_off,
+        slot_row_off, pair_row, row_pair, static_cast<uint4*>(xp), ctx->d_status);
+  } else {
+    rank_copy_kernel<false><<<tblocks, kThreads, 0, st>>>(
+        static_cast<const uint4*>(x), s.T, s.K, s.D / 8, topk_idx, R, s.E, s.S, Rcap, seg, nseg, hist, replicas, slot_off,
+        slot_row_off, pair_row, row_pair, static_cast<uint4*>(xp), ctx->d_status);
+  }
   MOEGPS_AFTER_LAUNCH(ctx);
   return MOEGPS_OK;
 }

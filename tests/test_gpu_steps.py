@@ -172,6 +172,8 @@ DISPATCH_CASES = [
     (256, 512, 8, 2, 8, 128, 1.0), (256, 512, 8, 2, 8, 1, 1.0), (1000, 256, 8, 2, 16, 128, 1.5),
     (777, 64, 64, 6, 80, 128, 1.2), (515, 128, 256, 8, 288, 128, 1.0), (515, 128, 256, 8, 288, 1, 1.0),
     (33, 64, 4, 4, 16, 4, 0.5), (1, 8, 1, 1, 1, 1, 0.0), (300, 72, 5, 1, 9, 32, 2.0), (0, 64, 4, 2, 6, 8, 1.0),
+    # more than 1024 segments of 256 pairs: the path that scans the segment counts on the device
+    (45000, 16, 16, 6, 20, 16, 1.0), (131073, 8, 3, 2, 7, 1, 0.7),
 ]
 
 
