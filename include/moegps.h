@@ -91,6 +91,14 @@ MOEGPS_API size_t moegps_workspace_bytes(const moegps_shape_t* shape);
 MOEGPS_API int moegps_route(moegps_ctx_t* ctx, const void* x, const void* w_router, const float* bias,
                  int32_t* topk_idx, float* topk_w, void* stream);
 
+/* route_histogram - moegps_route and moegps_histogram in one kernel: the router's epilogue also
+ * counts the selections per expert (the n_e of the paper's Eq. 1 with N = T*K), so the indices are
+ * not read back from memory and one launch is saved.  Same arguments and results as moegps_route,
+ * plus hist: int32 [E], fully overwritten (zeroed on the stream, then accumulated with integer
+ * atomics: exact and deterministic).  Bit-identical to moegps_route followed by moegps_histogram. */
+MOEGPS_API int moegps_route_histogram(moegps_ctx_t* ctx, const void* x, const void* w_router, const float* bias,
+                                      int32_t* topk_idx, float* topk_w, int32_t* hist, void* stream);
+
 /* Debug companion of moegps_route: also stores the fp32 logits (fp32 [T,E]) the selection was made on. */
 MOEGPS_API int moegps_route_logits(moegps_ctx_t* ctx, const void* x, const void* w_router, const float* bias,
                         float* logits, void* stream);

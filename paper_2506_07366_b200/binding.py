@@ -53,7 +53,7 @@ ERR_STATIC_SCRATCH_EXCEEDED = -9
 
 EXPORTS = (
     "moegps_create", "moegps_destroy", "moegps_rcap", "moegps_workspace_bytes", "moegps_route",
-    "moegps_route_logits", "moegps_histogram", "moegps_plan", "moegps_dispatch", "moegps_dispatch_static",
+    "moegps_route_histogram", "moegps_route_logits", "moegps_histogram", "moegps_plan", "moegps_dispatch", "moegps_dispatch_static",
     "moegps_expert_ffn", "moegps_expert_ffn_gate_up", "moegps_expert_ffn_down", "moegps_combine",
     "moegps_status", "moegps_launch_count", "moegps_last_cuda_error", "moegps_error_string",
     "moegps_selftest_bounded_wait", "moegps_predictor_update", "moegps_error_rate",
@@ -94,6 +94,7 @@ def _lib():
         "moegps_rcap": (i64, [ctypes.POINTER(moegps_shape_t)]),
         "moegps_workspace_bytes": (ctypes.c_size_t, [ctypes.POINTER(moegps_shape_t)]),
         "moegps_route": (ctypes.c_int, [vp] * 7),
+        "moegps_route_histogram": (ctypes.c_int, [vp] * 8),
         "moegps_route_logits": (ctypes.c_int, [vp] * 6),
         "moegps_histogram": (ctypes.c_int, [vp] * 4),
         "moegps_plan": (ctypes.c_int, [vp, vp, i32, vp, vp, vp, vp, vp]),
@@ -183,6 +184,16 @@ class Context:
             _ptr(bias, torch.float32, (s.E,), "bias", allow_none=True),
             _ptr(topk_idx, torch.int32, (s.T, s.K), "topk_idx"),
             _ptr(topk_w, torch.float32, (s.T, s.K), "topk_w"), _stream(stream)), "moegps_route")
+
+    def route_histogram(self, x, w_router, bias, topk_idx, topk_w, hist, stream=None):
+        s = self.shape
+        self._check(_lib().moegps_route_histogram(
+            self._h, _ptr(x, torch.bfloat16, (s.T, s.D), "x"),
+            _ptr(w_router, torch.bfloat16, (s.E, s.D), "w_router"),
+            _ptr(bias, torch.float32, (s.E,), "bias", allow_none=True),
+            _ptr(topk_idx, torch.int32, (s.T, s.K), "topk_idx"),
+            _ptr(topk_w, torch.float32, (s.T, s.K), "topk_w"),
+            _ptr(hist, torch.int32, (s.E,), "hist"), _stream(stream)), "moegps_route_histogram")
 
     def route_logits(self, x, w_router, bias, logits, stream=None):
         s = self.shape

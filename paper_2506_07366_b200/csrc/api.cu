@@ -93,7 +93,18 @@ int moegps_route(moegps_ctx_t* ctx, const void* x, const void* w_router, const f
   if (ctx->shape.T == 0) return MOEGPS_OK;          // nothing to route (empty tensors have no address)
   if (!all_ok(x, w_router, topk_idx, topk_w)) return MOEGPS_ERR_INVALID_ARG;
   if (bias && (reinterpret_cast<uintptr_t>(bias) & 3u)) return MOEGPS_ERR_INVALID_ARG;
-  return moegps_launch_route(ctx, x, w_router, bias, topk_idx, topk_w, nullptr, (cudaStream_t)stream);
+  return moegps_launch_route(ctx, x, w_router, bias, topk_idx, topk_w, nullptr, nullptr, (cudaStream_t)stream);
+}
+
+int moegps_route_histogram(moegps_ctx_t* ctx, const void* x, const void* w_router, const float* bias,
+                           int32_t* topk_idx, float* topk_w, int32_t* hist, void* stream) {
+  if (!ctx || !all_ok(hist)) return MOEGPS_ERR_INVALID_ARG;
+  if (ctx->shape.T == 0)                            // no tokens: the histogram is all zero
+    return cudaMemsetAsync(hist, 0, sizeof(int32_t) * ctx->shape.E, (cudaStream_t)stream) == cudaSuccess
+               ? MOEGPS_OK : MOEGPS_ERR_CUDA;
+  if (!all_ok(x, w_router, topk_idx, topk_w)) return MOEGPS_ERR_INVALID_ARG;
+  if (bias && (reinterpret_cast<uintptr_t>(bias) & 3u)) return MOEGPS_ERR_INVALID_ARG;
+  return moegps_launch_route(ctx, x, w_router, bias, topk_idx, topk_w, nullptr, hist, (cudaStream_t)stream);
 }
 
 int moegps_route_logits(moegps_ctx_t* ctx, const void* x, const void* w_router, const float* bias,
@@ -102,7 +113,7 @@ int moegps_route_logits(moegps_ctx_t* ctx, const void* x, const void* w_router, 
   if (ctx->shape.T == 0) return MOEGPS_OK;
   if (!all_ok(x, w_router, logits)) return MOEGPS_ERR_INVALID_ARG;
   if (bias && (reinterpret_cast<uintptr_t>(bias) & 3u)) return MOEGPS_ERR_INVALID_ARG;
-  return moegps_launch_route(ctx, x, w_router, bias, nullptr, nullptr, logits, (cudaStream_t)stream);
+  return moegps_launch_route(ctx, x, w_router, bias, nullptr, nullptr, logits, nullptr, (cudaStream_t)stream);
 }
 
 int moegps_histogram(moegps_ctx_t* ctx, const int32_t* topk_idx, int32_t* hist, void* stream) {

@@ -68,7 +68,7 @@ constexpr int kSegPairs = 256;
 
 // Per-step launchers (each validates nothing: the C entry points in api.cu do that).
 int moegps_launch_route(moegps_ctx* ctx, const void* x, const void* wr, const float* bias,
-                        int32_t* topk_idx, float* topk_w, float* logits_out, cudaStream_t st);
+                        int32_t* topk_idx, float* topk_w, float* logits_out, int32_t* hist, cudaStream_t st);
 int moegps_launch_histogram(moegps_ctx* ctx, const int32_t* topk_idx, int32_t* hist, cudaStream_t st);
 int moegps_launch_plan(moegps_ctx* ctx, const int32_t* pred, int32_t* replicas, int32_t* slot_off,
                        int32_t* slot_expert, int32_t* bound, cudaStream_t st);

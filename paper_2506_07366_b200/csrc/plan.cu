@@ -8,35 +8,33 @@ namespace {
 
 constexpr int kPlanThreads = 256;   // >= the largest supported E
 
+// A candidate in two 32-bit registers (the rounds are a chain of shuffles, so every register
+// counts): n = predicted count, re = (replicas << 12) | expert, kNone = not eligible.
+// (replicas <= 1024 and expert < 288 fit 11 + 12 bits; comparing `re` compares replicas first,
+// then the expert index - exactly the order in which equal ratios are resolved.)
 struct Cand {
-  long long n;   // predicted count; -1 marks "not eligible"
-  int r;
-  int e;
+  uint32_t n;
+  uint32_t re;
 };
+constexpr uint32_t kNone = 0xffffffffu;
 
-// Strict order of Algorithm 1's choice: larger n/r first, then fewer replicas, then lower index.
+// Strict order of Algorithm 1's choice: larger n/r first (exact: 64-bit cross-multiplication),
+// then fewer replicas, then lower index.
 __device__ __forceinline__ bool better(const Cand& a, const Cand& b) {
-  if (a.n < 0) return false;
-  if (b.n < 0) return true;
-  const long long lhs = a.n * (long long)b.r;
-  const long long rhs = b.n * (long long)a.r;
+  if (a.re == kNone) return false;
+  if (b.re == kNone) return true;
+  const unsigned long long lhs = (unsigned long long)a.n * (b.re >> 12);
+  const unsigned long long rhs = (unsigned long long)b.n * (a.re >> 12);
   if (lhs != rhs) return lhs > rhs;
-  if (a.r != b.r) return a.r < b.r;
-  return a.e < b.e;
-}
-
-__device__ __forceinline__ Cand shfl_xor(const Cand& c, int m) {
-  Cand o;
-  o.n = __shfl_xor_sync(0xffffffffu, c.n, m);
-  o.r = __shfl_xor_sync(0xffffffffu, c.r, m);
-  o.e = __shfl_xor_sync(0xffffffffu, c.e, m);
-  return o;
+  return a.re < b.re;
 }
 
 __device__ __forceinline__ Cand warp_best(Cand c) {
 #pragma unroll
   for (int m = 16; m >= 1; m >>= 1) {
-    const Cand o = shfl_xor(c, m);
+    Cand o;
+    o.n = __shfl_xor_sync(0xffffffffu, c.n, m);
+    o.re = __shfl_xor_sync(0xffffffffu, c.re, m);
     if (better(o, c)) c = o;
   }
   return c;
@@ -63,31 +61,32 @@ plan_kernel(const int32_t* __restrict__ pred, int E, int S, int c_max, int32_t* 
   // l, l+32, ... in registers, picks its best candidate, and a shuffle butterfly picks the winner.
   if (warp == 0) {
     constexpr int kPerLane = kPlanThreads / 32;
-    long long ln[kPerLane];
-    int lr[kPerLane];
+    uint32_t ln[kPerLane];
+    int lr[kPerLane];            // 0 = no such expert
 #pragma unroll
     for (int i = 0; i < kPerLane; ++i) {
       const int e = lane + 32 * i;
       const int v = e < E ? pred[e] : 0;
-      ln[i] = e < E ? (v < 0 ? 0 : v) : -1;
+      ln[i] = v < 0 ? 0u : (uint32_t)v;
       lr[i] = e < E ? 1 : 0;
     }
     for (int round = 0; round < S - E; ++round) {
       Cand c;
-      c.n = -1; c.r = 0; c.e = kPlanThreads + lane;
+      c.n = 0; c.re = kNone;
 #pragma unroll
       for (int i = 0; i < kPerLane; ++i) {
         Cand d;
-        d.n = (ln[i] >= 0 && (c_max <= 0 || lr[i] < c_max)) ? ln[i] : -1;
-        d.r = lr[i];
-        d.e = lane + 32 * i;
+        d.n = ln[i];
+        d.re = (lr[i] > 0 && (c_max <= 0 || lr[i] < c_max)) ? (((uint32_t)lr[i] << 12) | (uint32_t)(lane + 32 * i))
+                                                            : kNone;
         if (better(d, c)) c = d;
       }
       c = warp_best(c);
-      if (c.n < 0) break;          // nobody may take another copy: the remaining slots stay empty
+      if (c.re == kNone) break;    // nobody may take another copy: the remaining slots stay empty
+      const int win = (int)(c.re & 0xfffu);
 #pragma unroll
       for (int i = 0; i < kPerLane; ++i)
-        if (c.e == lane + 32 * i) lr[i] += 1;
+        if (win == lane + 32 * i) lr[i] += 1;
     }
 #pragma unroll
     for (int i = 0; i < kPerLane; ++i) plan_r[lane + 32 * i] = lr[i];

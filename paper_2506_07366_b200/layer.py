@@ -46,14 +46,13 @@ class MoeLayer:
         self._planned = True
 
     def forward(self, x, stream=None, out=None):
-        """route -> histogram -> dispatch -> expert_ffn -> combine on device tensor x [T, D].
+        """route + histogram (one kernel) -> dispatch -> expert_ffn -> combine on device tensor x [T, D].
         The result goes to `out` (bf16 [T, D]) if given, else to the layer's own buffer."""
         if not self._planned:
             raise RuntimeError("call plan(predicted_hist) before forward()")
         c = self.ctx
         out = self.out if out is None else out
-        c.route(x, self.w_router, self.bias, self.topk_idx, self.topk_w, stream)
-        c.histogram(self.topk_idx, self.hist, stream)
+        c.route_histogram(x, self.w_router, self.bias, self.topk_idx, self.topk_w, self.hist, stream)
         c.dispatch(x, self.topk_idx, self.hist, self.replicas, self.slot_off, self.slot_row_off,
                    self.row_pair, self.pair_row, self.xp, self.workspace, stream)
         c.expert_ffn(self.xp, self.slot_row_off, self.slot_expert, self.w_gate, self.w_up,

@@ -67,6 +67,14 @@ def test_route(w):
     hz.assert_close_rel_max(got_w, ref_w, "topk_w")
     assert np.abs(got_w - ref_w).max() < 2e-5
     assert np.abs(got_w.sum(axis=1) - 1).max() < 1e-5
+    # the fused call (router epilogue also counts the selections): same indices and weights bit for
+    # bit, histogram equal to the oracle's, on two calls in a row (the counters start from zero each time)
+    for _ in range(2):
+        idx2, wt2, hist = poison_i32(w.T, w.K), torch.full_like(wt, float("nan")), poison_i32(w.E)
+        ctx.route_histogram(xd, wrd, bd, idx2, wt2, hist)
+        ctx.check_status()
+        assert torch.equal(idx2, idx) and torch.equal(wt2, wt)
+        assert np.array_equal(hist.cpu().numpy(), oracle.histogram(ref_idx, w.E))
 
 
 def test_route_no_bias_and_exact_ties():
