@@ -190,3 +190,17 @@ def test_layer_full_size_sampled(name):
     out_got = out[torch.from_numpy(tokens).to(DEV).long()].float().cpu().numpy()
     hz.assert_close_rel_max(out_got, out_ref[tokens], "out (sampled tokens)")
     assert torch.isfinite(out.float()).all()
+
+
+def test_plan_study_runs_on_a_small_workload():
+    """The plan-quality script end to end on the tiny workload: more replica slots never raise the
+    bottleneck load under an exact prediction, and the reported loads respect the planner's bound."""
+    from paper_2506_07366_b200 import plan_study
+    rows = plan_study.study("tiny", extras=[0, 2, 4], noises=[0.0])
+    assert [r["slots"] for r in rows] == [8, 10, 12]
+    loads = [r["max_slot_load"] for r in rows]
+    assert loads == sorted(loads, reverse=True)
+    for r in rows:
+        assert r["max_slot_load"] == r["plan_bound"]          # exact prediction: the split realises the plan
+        assert r["prediction_error_rate"] == 0.0
+        assert r["ffn_ms_bottleneck"] > 0 and r["ffn_ms_even_share"] > 0
