@@ -262,6 +262,7 @@ def run_ours(args):
     achieved = flops_gate_up / (gate_up_ms * 1e-3) / 1e12
     ffn_tflops = 6.0 * w.R * w.D * w.F / ((gate_up_ms + down_ms) * 1e-3) / 1e12
     hist_np = true_hist.numpy().astype("float64")
+    active = int((hist_np > 0).sum())
     # slot loads of the last step: rows that carry a pair, counted per slot
     occupied = (layer.row_pair >= 0).to(torch.int64).cumsum(0)
     ends = layer.slot_row_off[1:].long().clamp(max=shape.Rcap) - 1
@@ -302,7 +303,14 @@ def run_ours(args):
                      "peak_source": peaks["source"] + peak_kind,
                      "ms_per_launch": gate_up_ms, "traffic": GATE_UP_DRAM_TRAFFIC.get(w.name)},
         "expert_ffn": {"tflops": ffn_tflops, "gate_up_ms": gate_up_ms, "down_ms": down_ms,
-                       "frac_of_sustained_peak": ffn_tflops / peaks["bf16_sustained"]},
+                       "frac_of_sustained_peak": ffn_tflops / peaks["bf16_sustained"],
+                       # the other roof of the grouped GEMMs: every expert that received tokens has its
+                       # weights streamed from HBM once per GEMM (binding when slots hold few rows)
+                       "active_experts": active,
+                       "gate_up_weight_gbs": active * 2.0 * w.D * w.F * 2 / (gate_up_ms * 1e-3) / 1e9,
+                       "down_weight_gbs": active * 1.0 * w.D * w.F * 2 / (down_ms * 1e-3) / 1e9,
+                       "gate_up_weight_frac_of_hbm_peak":
+                           active * 2.0 * w.D * w.F * 2 / (gate_up_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
     }
     if kernels is not None:
         line["calls_cold_l2"] = kernels
