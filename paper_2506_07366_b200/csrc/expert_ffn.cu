@@ -7,13 +7,8 @@
 // warps 2..9 = epilogue (two per quarter of the 128 TMEM lanes, half the columns each).  A 4-stage ring
 // (TMA -> tcgen05.mma) and two TMEM accumulators (mainloop of tile i+1 overlaps the epilogue of tile
 // i) are handed around with mbarriers; every wait is bounded and raises an abort flag on expiry.
-// Tiles are enumerated on the device from slot_row_off (no host round trip).  Within a slot the
-// order is column tile, then row tile, so that CTAs working at the same time share weight tiles in
-// L2.  Slots with several row tiles (their tiles re-use a weight tile from L2 and run at the tensor
-// core's pace) and slots with one row tile (every tile streams its own weights from HBM) are kept
-// in two lists, and every round of gridDim.x tiles takes its share of both: HBM streaming and
-// tensor work then overlap instead of alternating in phases (measured: -5 % step time on the
-// 256-expert workload, neutral where every slot is large).
+// Tiles are enumerated on the device from slot_row_off (no host round trip): slot-major, then
+// column tile, then row tile, so that CTAs working at the same time share weight tiles in L2.
 #include "common.cuh"
 #include "sm100.cuh"
 
@@ -40,13 +35,9 @@ constexpr int kMaxS = 1024;
 constexpr int kTmemCols = 512;
 
 struct __align__(16) Tables {
-  int32_t tile_base[kMaxS + 1];    // first tile index of each listed slot, in list order
+  int32_t tile_base[kMaxS + 1];    // first tile index of each slot
   int32_t row_off[kMaxS + 1];
-  int16_t expert[kMaxS];
-  int16_t order[kMaxS];            // listed slots: those with several row tiles first, then the single-tile ones
-  int32_t n_listed;                // slots that have rows and a valid expert
-  int32_t tiles_multi, tiles_single;   // tiles of the two lists
-  int32_t per_round_multi, per_round_single, mixed_rounds, round_tiles;
+  int32_t expert[kMaxS];
 };
 
 constexpr int kEpilogueWarps = 8;
@@ -60,42 +51,25 @@ struct TileCoord {
   int expert;
 };
 
-// tile number within the slot list -> coordinates
-__device__ __forceinline__ TileCoord decode_listed(const Tables& tb, int idx, int n_tiles) {
-  int lo = 0, hi = tb.n_listed;       // find i with tile_base[i] <= idx < tile_base[i+1]
+__device__ __forceinline__ TileCoord decode_tile_rows(const Tables& tb, int S, int tile, int n_tiles, int tile_rows) {
+  int lo = 0, hi = S;                 // find s with tile_base[s] <= tile < tile_base[s+1]
   while (hi - lo > 1) {
     const int mid = (lo + hi) >> 1;
-    if (tb.tile_base[mid] <= idx) lo = mid; else hi = mid;
+    if (tb.tile_base[mid] <= tile) lo = mid; else hi = mid;
   }
-  const int s = tb.order[lo];
-  const int local = idx - tb.tile_base[lo];
-  const int mt = (tb.tile_base[lo + 1] - tb.tile_base[lo]) / n_tiles;   // row tiles of this slot
+  const int s = lo;
+  const int local = tile - tb.tile_base[s];
+  const int mt = (tb.tile_base[s + 1] - tb.tile_base[s]) / n_tiles;   // row tiles of this slot
   TileCoord c;
   c.n_tile = local / mt;
-  c.m0 = tb.row_off[s] + (local % mt) * BM;
+  c.m0 = tb.row_off[s] + (local % mt) * tile_rows;
   c.row_end = tb.row_off[s + 1];
   c.expert = tb.expert[s];
   return c;
 }
 
-// `tile` = position in the processing order (CTA c takes c, c + gridDim.x, ...).  The first
-// `mixed_rounds` rounds of `round_tiles` tiles hold `per_round_multi` tiles of the multi-row-tile list
-// (kept consecutive: the row tiles of one column tile stay together) and `per_round_single` of the
-// other; the window of multi tiles moves by its own width from round to round so that every CTA gets
-// the same mix.  What is left of either list follows in list order.
-__device__ __forceinline__ TileCoord decode_tile(const Tables& tb, int tile, int n_tiles) {
-  const int w = tb.round_tiles, a = tb.per_round_multi, b = tb.per_round_single;
-  int idx;
-  if (tile < tb.mixed_rounds * w) {
-    const int round = tile / w;
-    const int r = (tile - round * w + round * a) % w;
-    idx = r < a ? round * a + r : tb.tiles_multi + round * b + (r - a);
-  } else {
-    const int t2 = tile - tb.mixed_rounds * w;
-    const int left_multi = tb.tiles_multi - tb.mixed_rounds * a;
-    idx = t2 < left_multi ? tb.mixed_rounds * a + t2 : tb.tiles_multi + tb.mixed_rounds * b + (t2 - left_multi);
-  }
-  return decode_listed(tb, idx, n_tiles);
+__device__ __forceinline__ TileCoord decode_tile(const Tables& tb, int S, int tile, int n_tiles) {
+  return decode_tile_rows(tb, S, tile, n_tiles, BM);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -192,10 +166,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
 
   // ---------------------------------------------------------------- set-up
   for (int s = threadIdx.x; s <= S; s += kThreads) tb.row_off[s] = slot_row_off[s];
-  for (int s = threadIdx.x; s < S; s += kThreads) {
-    const int e = slot_expert[s];
-    tb.expert[s] = (int16_t)(e < -1 || e > 32767 ? 32767 : e);   // out-of-range values stay out of range
-  }
+  for (int s = threadIdx.x; s < S; s += kThreads) tb.expert[s] = slot_expert[s];
   if (threadIdx.x == 0) {
     for (int i = 0; i < kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 8); }
@@ -211,36 +182,15 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
   }
   __syncthreads();
   if (threadIdx.x == 0) {
-    int acc = 0, n = 0;
-    for (int pass = 0; pass < 2; ++pass) {        // pass 0 lists the slots with several row tiles
-      for (int s = 0; s < S; ++s) {
-        const int rows = tb.row_off[s + 1] - tb.row_off[s];
-        const int e = tb.expert[s];
-        if (rows > 0 && e >= 0 && e < E) {
-          const int mt = (rows + BM - 1) / BM;
-          if ((mt > 1) == (pass == 0)) {
-            tb.tile_base[n] = acc;
-            tb.order[n] = (int16_t)s;
-            acc += mt * n_tiles;
-            ++n;
-          }
-        } else if (pass == 0 && rows > 0 && e >= E) {
-          moegps_report(status, MOEGPS_ERR_BAD_INDEX, s);
-        }
-      }
-      if (pass == 0) tb.tiles_multi = acc;
+    int acc = 0;
+    for (int s = 0; s < S; ++s) {
+      tb.tile_base[s] = acc;
+      const int rows = tb.row_off[s + 1] - tb.row_off[s];
+      const int e = tb.expert[s];
+      if (rows > 0 && e >= 0 && e < E) acc += ((rows + BM - 1) / BM) * n_tiles;
+      else if (rows > 0 && e >= E) moegps_report(status, MOEGPS_ERR_BAD_INDEX, s);
     }
-    tb.tile_base[n] = acc;
-    tb.n_listed = n;
-    tb.tiles_single = acc - tb.tiles_multi;
-    const int w = (int)gridDim.x;
-    int a = acc > 0 ? (int)(((long long)w * tb.tiles_multi + acc / 2) / acc) : 0;   // share of a round
-    if (tb.tiles_multi > 0 && a == 0) a = 1;
-    if (tb.tiles_single > 0 && a == w) a = w - 1;
-    tb.per_round_multi = a;
-    tb.per_round_single = w - a;
-    tb.round_tiles = w;
-    tb.mixed_rounds = (a > 0 && a < w) ? min(tb.tiles_multi / a, tb.tiles_single / (w - a)) : 0;
+    tb.tile_base[S] = acc;
     *total_tiles_p = acc;
   }
   tc_fence_before_sync();
@@ -256,7 +206,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
       uint32_t phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-        const TileCoord tc = decode_tile(tb, tile, n_tiles);
+        const TileCoord tc = decode_tile(tb, S, tile, n_tiles);
         const int nb0 = tc.n_tile * cols_per_tile;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -314,7 +264,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     uint32_t acc_phase = 0;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-      const TileCoord tc = decode_tile(tb, tile, n_tiles);
+      const TileCoord tc = decode_tile(tb, S, tile, n_tiles);
       if (!mbar_wait(&acc_full[acc], acc_phase, abort_flag, 256)) { ok = false; break; }
       tc_fence_after_sync();
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * BNACC;
