@@ -32,7 +32,8 @@ UNIT = "tokens/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one gate+up GEMM launch, from the ncu captures
 # summarised under profiles/ (bytes; None = not captured for the current kernel)
-GATE_UP_DRAM_TRAFFIC = {"mixtral": 2064364288 + 241741568}   # profiles/ncu_traffic_mixtral.md
+GATE_UP_DRAM_TRAFFIC = {"mixtral": 2064364288 + 241741568,          # profiles/ncu_traffic_mixtral.md
+                        "fine_grained": 13879219968 + 228023552}    # profiles/ncu_traffic_fine_grained.md
 
 
 # ------------------------------------------------------------------------------------- helpers
