@@ -1,17 +1,25 @@
 #!/usr/bin/env python
-"""Benchmark of the MoE hot path (route -> histogram -> plan -> dispatch -> expert_ffn -> combine).
+"""Benchmark of the MoE hot path (plan -> route + histogram -> dispatch -> expert_ffn -> combine).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
 
 One "step" is one pass of the whole path over one batch of the workload.  Prints ONE JSON line.
+The default workload is `mixtral_skew` (Mixtral-8x7B layer shape, 16384 tokens, heavy routing skew,
+16 slots for 8 experts, noisy predicted histogram): the largest single-GPU configuration, and one in
+which the duplication plan really replicates experts inside the timed step.  The other full-size
+workloads are measured after it in the same process and reported in the `per_workload` block.
 With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank runs the same workload
 on its own batch: batches are independent, so there is no data-path collective ("weak" scaling);
 the only communication is the barrier and the max-over-ranks of the elapsed time.
 `--impl reference` times the CPU oracle on a bounded sample of the same workload.
+`--record-traffic CSV` (no GPU needed) turns an `ncu --csv` capture of the DRAM byte counters into
+profiles/dram_traffic.json, the file the `roofline.traffic` figure is read from.
 """
 from __future__ import annotations
 
 import argparse
+import csv
+import hashlib
 import json
 import os
 import statistics
@@ -29,11 +37,10 @@ from paper_2506_07366_b200 import workloads as wl  # noqa: E402
 
 METRIC = "moe_layer_tokens_per_s"
 UNIT = "tokens/s"
-
-# dram__bytes_read.sum + dram__bytes_write.sum of one gate+up GEMM launch, from the ncu captures
-# summarised under profiles/ (bytes; None = not captured for the current kernel)
-GATE_UP_DRAM_TRAFFIC = {"mixtral": 2064364288 + 241741568,          # profiles/ncu_traffic_mixtral.md
-                        "fine_grained": 13879219968 + 228023552}    # profiles/ncu_traffic_fine_grained.md
+DEFAULT_WORKLOAD = "mixtral_skew"
+OTHER_WORKLOADS = ("mixtral", "many_expert", "fine_grained")
+TRAFFIC_JSON = os.path.join(ROOT, "profiles", "dram_traffic.json")
+GEMM_SOURCES = ("expert_ffn.cu", "sm100.cuh")       # what the captured DRAM traffic depends on
 
 
 # ------------------------------------------------------------------------------------- helpers
@@ -45,6 +52,68 @@ def measured_peaks():
         return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_burst=float(p["bf16_tflops"]),
                     bf16_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
     return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+def gemm_source_hash() -> str:
+    h = hashlib.sha256()
+    for name in GEMM_SOURCES:
+        with open(os.path.join(ROOT, "paper_2506_07366_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(workload: str, pairs: int):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one gate+up GEMM launch of `workload`, from
+    the ncu capture recorded in profiles/dram_traffic.json; None when there is no capture or the
+    kernel's sources have changed since it was taken.  A capture of a reduced cut of the workload
+    (fewer routed pairs, same layer) is scaled to a full launch by the pairs processed."""
+    try:
+        with open(TRAFFIC_JSON) as f:
+            rec = json.load(f)["gate_up"][workload]
+    except (OSError, KeyError, ValueError):
+        return None
+    if rec.get("source_hash") != gemm_source_hash():
+        return None
+    return (rec["dram_read_bytes"] + rec["dram_write_bytes"]) * (pairs / rec["pairs_in_capture"])
+
+
+def record_traffic(csv_path: str, workload: str, pairs: int):
+    """Reads an `ncu --csv` log that holds dram__bytes_read.sum / dram__bytes_write.sum of
+    grouped_gemm_kernel launches and stores the per-launch mean of the gate+up and the down GEMM."""
+    rows = []
+    with open(csv_path, newline="") as f:
+        lines = [ln for ln in f if ln.startswith('"')]
+    for r in csv.DictReader(lines):
+        rows.append(r)
+    out = {}
+    for key, tag in (("gate_up", "grouped_gemm_kernel<1>"), ("down", "grouped_gemm_kernel<0>")):
+        acc = {"dram__bytes_read.sum": [], "dram__bytes_write.sum": []}
+        for r in rows:
+            if tag not in r.get("Kernel Name", ""):
+                continue
+            m = r.get("Metric Name")
+            if m in acc:
+                v = float(r["Metric Value"].replace(",", ""))
+                unit = r.get("Metric Unit", "byte").lower()
+                v *= {"byte": 1.0, "kbyte": 1e3, "mbyte": 1e6, "gbyte": 1e9}.get(unit, 1.0)
+                acc[m].append(v)
+        if acc["dram__bytes_read.sum"]:
+            out[key] = {"dram_read_bytes": statistics.mean(acc["dram__bytes_read.sum"]),
+                        "dram_write_bytes": statistics.mean(acc["dram__bytes_write.sum"]),
+                        "launches": len(acc["dram__bytes_read.sum"]), "pairs_in_capture": pairs,
+                        "source_hash": gemm_source_hash()}
+    if not out:
+        raise SystemExit(f"{csv_path}: no grouped_gemm_kernel DRAM counters found")
+    data = {}
+    if os.path.exists(TRAFFIC_JSON):
+        with open(TRAFFIC_JSON) as f:
+            data = json.load(f)
+    for key, rec in out.items():
+        data.setdefault(key, {})[workload] = rec
+    with open(TRAFFIC_JSON, "w") as f:
+        json.dump(data, f, indent=1, sort_keys=True)
+        f.write("\n")
+    print(json.dumps(out))
 
 
 class ClockSampler:
@@ -130,10 +199,222 @@ def whole_job_rate(world: int, tokens_per_rank: int, steps: int, elapsed_ms: flo
 
 
 # ------------------------------------------------------------------------------------- our arm
-def run_ours(args):
-    from paper_2506_07366_b200 import binding
-    from paper_2506_07366_b200.layer import MoeLayer
+class Bench:
+    """One workload resident on the device: layer, inputs, prediction."""
 
+    A = 128
+
+    def __init__(self, w, rank: int, local_rank: int):
+        from paper_2506_07366_b200 import binding
+        from paper_2506_07366_b200.layer import MoeLayer
+        self.w, self.dev = w, torch.device("cuda", local_rank)
+        dev = self.dev
+        self.shape = binding.Shape(w.T, w.D, w.F, w.E, w.K, w.S, w.gate_mode, self.A)
+        # every rank draws its own batch (same weights: data parallel replicas of the layer)
+        self.wr, self.bias = wl.router(w, dev)
+        self.w1, self.w3, self.w2 = wl.expert_weights(w, dev)
+        self.x = wl.activations(rank_workload(w, rank), dev)
+        self.layer = layer = MoeLayer(self.shape, self.wr, self.bias, self.w1, self.w3, self.w2, device=local_rank)
+        self.ctx = ctx = layer.ctx
+        # the workload's stand-in for the predictor: computed once, outside the timed region, with the
+        # library's own route + histogram (the prediction is an INPUT of the path)
+        ctx.route(self.x, self.wr, self.bias, layer.topk_idx, layer.topk_w)
+        ctx.histogram(layer.topk_idx, layer.hist)
+        self.true_hist = layer.hist.cpu()
+        if w.prediction == "true":
+            pred = self.true_hist.clone()
+        elif w.prediction == "noisy":
+            pred = wl.noisy_prediction(w, self.true_hist)
+        else:
+            xprev = wl.activations(w, dev, previous=True)
+            ctx.route(xprev, self.wr, self.bias, layer.topk_idx, layer.topk_w)
+            ctx.histogram(layer.topk_idx, layer.hist)
+            pred = layer.hist.cpu().clone()
+        self.pred = pred
+        self.pred_dev = pred.to(dev, torch.int32)
+        self.gemm_marks = []
+
+    def step(self, record: bool):
+        L, c, w = self.layer, self.ctx, self.w
+        c.plan(self.pred_dev, w.S, L.replicas, L.slot_off, L.slot_expert, L.bound)
+        c.route_histogram(self.x, self.wr, self.bias, L.topk_idx, L.topk_w, L.hist)     # route + histogram fused
+        c.dispatch(self.x, L.topk_idx, L.hist, L.replicas, L.slot_off, L.slot_row_off, L.row_pair, L.pair_row,
+                   L.xp, L.workspace)
+        stream = torch.cuda.current_stream()
+        if record:
+            a, b, e = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            a.record(stream)
+        c.expert_ffn_gate_up(L.xp, L.slot_row_off, L.slot_expert, self.w1, self.w3, L.h_ws)
+        if record:
+            b.record(stream)
+        c.expert_ffn_down(L.h_ws, L.slot_row_off, L.slot_expert, self.w2, L.yp)
+        if record:
+            e.record(stream)
+            self.gemm_marks.append((a, b, e))
+        c.combine(L.yp, L.pair_row, L.topk_w, L.out)
+
+    def timed_steps(self, steps: int, warmup: int, barrier):
+        """W warm-up steps, then exactly `steps` steps between two events on the launching stream."""
+        stream = torch.cuda.current_stream()
+        for _ in range(warmup):
+            self.step(False)
+        barrier()
+        self.ctx.check_status()
+        self.gemm_marks = []
+        launches0 = self.ctx.launch_count()
+        barrier()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record(stream)
+        for _ in range(steps):
+            self.step(True)
+        t1.record(stream)
+        barrier()
+        self.ctx.check_status()
+        ms = t0.elapsed_time(t1)
+        gate_up = statistics.mean(a.elapsed_time(b) for a, b, _ in self.gemm_marks)
+        down = statistics.mean(b.elapsed_time(e) for _, b, e in self.gemm_marks)
+        return ms, gate_up, down, self.ctx.launch_count() - launches0
+
+    def e2e_steps(self, steps: int, warmup: int, barrier):
+        """End to end through the public layer API with pinned host buffers, copies inside the timing
+        (every step copies its batch in and its result out; HostPipeline overlaps the copies of
+        neighbouring steps with the compute, as a serving loop would)."""
+        from paper_2506_07366_b200.layer import HostPipeline
+        w, layer = self.w, self.layer
+        stream = torch.cuda.current_stream()
+        xh = [self.x.cpu().pin_memory() for _ in range(2)]
+        oh = [torch.empty(w.T, w.D, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
+        pipe = HostPipeline(layer, depth=2)
+        layer.plan(self.pred_dev)
+        for i in range(max(2, min(3, warmup))):
+            pipe.submit(xh[i % 2], oh[i % 2])
+        pipe.drain()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(steps):
+            layer.plan(self.pred_dev)
+            pipe.submit(xh[i % 2], oh[i % 2])
+        pipe.drain()
+        e1.record(stream)
+        barrier()
+        self.ctx.check_status()
+        return e0.elapsed_time(e1)
+
+    def load_statistics(self) -> dict:
+        """The paper's load statistics of the last batch, from the library's own outputs: skewness
+        before and after duplication, the planner's bound, the prediction's error rate."""
+        w, layer = self.w, self.layer
+        hist = self.true_hist.numpy().astype("float64")
+        occupied = (layer.row_pair >= 0).to(torch.int64).cumsum(0)
+        ends = layer.slot_row_off[1:].long().clamp(max=self.shape.Rcap) - 1
+        starts = layer.slot_row_off[:-1].long() - 1
+        cum_at = lambda i: torch.where(i >= 0, occupied[i.clamp(min=0)], torch.zeros_like(i))  # noqa: E731
+        slot_loads = (cum_at(ends) - cum_at(starts)).cpu().numpy()
+        err_dev = torch.zeros(1, dtype=torch.float64, device=self.dev)
+        self.ctx.error_rate(self.pred_dev, layer.hist, err_dev)
+        return {"skewness": float(hist.max() / (hist.sum() / w.E)),
+                "skewness_after_plan": float(slot_loads.max() / (w.R / w.S)),
+                "max_slot_load": int(slot_loads.max()), "plan_bound": int(layer.bound.item()),
+                "prediction_error_rate": float(err_dev.item()), "active_experts": int((hist > 0).sum()),
+                "max_replicas": int(layer.replicas.max().item())}
+
+    def per_call_timings(self, peaks, iters=7):
+        """Each library call timed alone (CUDA events on the launching stream, median of `iters`) with
+        a cold L2: before every call a 512 MB buffer is READ, which leaves L2 full of clean lines of
+        that buffer, so the call's inputs come from HBM and its stores evict nothing dirty.  The
+        interval between the two events also holds the launch latency of the stream and the event
+        records themselves (`event_pair` = the same measurement with nothing in between; calls that
+        launch two kernels pay the gap twice).  These numbers explain the step time; they are not
+        part of the timed step."""
+        w, L, c = self.w, self.layer, self.ctx
+        stream = torch.cuda.current_stream()
+        evict = torch.zeros(128 << 20, dtype=torch.float32, device=self.dev)
+        R, T, D, F, E, K = w.R, w.T, w.D, w.F, w.E, w.K
+        c.plan(self.pred_dev, w.S, L.replicas, L.slot_off, L.slot_expert, L.bound)
+        calls = [
+            ("plan", lambda: c.plan(self.pred_dev, w.S, L.replicas, L.slot_off, L.slot_expert, L.bound), None, None),
+            ("route", lambda: c.route(self.x, self.wr, self.bias, L.topk_idx, L.topk_w),
+             2.0 * T * D + 2.0 * E * D + 8.0 * T * K, 2.0 * T * D * E),
+            ("histogram", lambda: c.histogram(L.topk_idx, L.hist), 4.0 * R, None),
+            ("route_histogram", lambda: c.route_histogram(self.x, self.wr, self.bias, L.topk_idx, L.topk_w, L.hist),
+             2.0 * T * D + 2.0 * E * D + 8.0 * T * K, 2.0 * T * D * E),
+            ("dispatch", lambda: c.dispatch(self.x, L.topk_idx, L.hist, L.replicas, L.slot_off, L.slot_row_off,
+                                            L.row_pair, L.pair_row, L.xp, L.workspace),
+             2.0 * T * D + 2.0 * R * D + 12.0 * R, None),
+            ("expert_ffn_gate_up", lambda: c.expert_ffn_gate_up(L.xp, L.slot_row_off, L.slot_expert, self.w1, self.w3,
+                                                                L.h_ws), None, 4.0 * R * D * F),
+            ("expert_ffn_down", lambda: c.expert_ffn_down(L.h_ws, L.slot_row_off, L.slot_expert, self.w2, L.yp),
+             None, 2.0 * R * D * F),
+            ("combine", lambda: c.combine(L.yp, L.pair_row, L.topk_w, L.out), 2.0 * R * D + 2.0 * T * D + 8.0 * R, None),
+            ("event_pair", lambda: None, None, None),
+        ]
+        out = {}
+        for name, fn, nbytes, flops in calls:
+            times = []
+            for _ in range(iters):
+                evict.sum()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                fn()
+                b.record(stream)
+                b.synchronize()
+                times.append(a.elapsed_time(b))
+            ms = statistics.median(times)
+            rec = {"us": ms * 1e3}
+            if nbytes is not None:
+                rec["gbs"] = nbytes / (ms * 1e-3) / 1e9
+                rec["frac_of_hbm_peak"] = rec["gbs"] / peaks["hbm_gbs"]
+            if flops is not None and name.startswith("expert"):
+                rec["tflops"] = flops / (ms * 1e-3) / 1e12
+                rec["frac_of_burst_peak"] = rec["tflops"] / peaks["bf16_burst"]
+            out[name] = rec
+        c.check_status()
+        return out
+
+    def ffn_summary(self, gate_up_ms, down_ms, peaks, active) -> dict:
+        w = self.w
+        ffn_tflops = 6.0 * w.R * w.D * w.F / ((gate_up_ms + down_ms) * 1e-3) / 1e12
+        # the other roof of the grouped GEMMs: every expert that received tokens has its weights
+        # streamed from HBM once per GEMM, and the activations go in and out once (binding when
+        # slots hold few rows)
+        bytes_gate_up = active * 2.0 * w.D * w.F * 2 + 2.0 * w.R * w.D + 2.0 * w.R * w.F
+        bytes_down = active * 1.0 * w.D * w.F * 2 + 2.0 * w.R * w.F + 2.0 * w.R * w.D
+        return {"tflops": ffn_tflops, "gate_up_ms": gate_up_ms, "down_ms": down_ms,
+                "frac_of_burst_peak": ffn_tflops / peaks["bf16_burst"],
+                "frac_of_sustained_peak": ffn_tflops / peaks["bf16_sustained"],
+                "gate_up_frac_of_burst_peak": 4.0 * w.R * w.D * w.F / (gate_up_ms * 1e-3) / 1e12 / peaks["bf16_burst"],
+                "down_frac_of_burst_peak": 2.0 * w.R * w.D * w.F / (down_ms * 1e-3) / 1e12 / peaks["bf16_burst"],
+                "gate_up_hbm_gbs": bytes_gate_up / (gate_up_ms * 1e-3) / 1e9,
+                "down_hbm_gbs": bytes_down / (down_ms * 1e-3) / 1e9,
+                "gate_up_frac_of_hbm_peak": bytes_gate_up / (gate_up_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                "down_frac_of_hbm_peak": bytes_down / (down_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+
+    def close(self):
+        self.layer.ctx.close()
+
+
+def compact_record(b: Bench, peaks, steps: int, barrier) -> dict:
+    """The short form reported for the workloads other than the headline one."""
+    ms, gate_up, down, _ = b.timed_steps(steps, 3, barrier)
+    stats = b.load_statistics()
+    calls = b.per_call_timings(peaks, iters=5)
+    ffn = b.ffn_summary(gate_up, down, peaks, stats["active_experts"])
+    w = b.w
+    return {"T": w.T, "D": w.D, "F": w.F, "E": w.E, "K": w.K, "S": w.S, "steps": steps,
+            "ms_per_step": ms / steps, "tokens_per_s": w.T * steps / (ms * 1e-3),
+            "ffn_tflops": ffn["tflops"], "gate_up_ms": gate_up, "down_ms": down,
+            "gate_up_frac_of_burst_peak": ffn["gate_up_frac_of_burst_peak"],
+            "down_frac_of_burst_peak": ffn["down_frac_of_burst_peak"],
+            "gate_up_frac_of_hbm_peak": ffn["gate_up_frac_of_hbm_peak"],
+            "down_frac_of_hbm_peak": ffn["down_frac_of_hbm_peak"],
+            "cold_l2_us": {k: round(calls[k]["us"], 2) for k in ("route_histogram", "dispatch", "combine", "plan")},
+            "frac_of_hbm_peak": {k: round(calls[k]["frac_of_hbm_peak"], 3)
+                                 for k in ("route_histogram", "dispatch", "combine")},
+            "skewness": stats["skewness"], "skewness_after_plan": stats["skewness_after_plan"]}
+
+
+def run_ours(args):
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -148,108 +429,25 @@ def run_ours(args):
     if args.gpus != world:
         raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}: launch with torch.distributed.run")
 
-    w = wl.WORKLOADS[args.workload]
-    A = 128
-    shape = binding.Shape(w.T, w.D, w.F, w.E, w.K, w.S, w.gate_mode, A)
-    # every rank draws its own batch (same weights: data parallel replicas of the layer)
-    wr, bias = wl.router(w, dev)
-    w1, w3, w2 = wl.expert_weights(w, dev)
-    x = wl.activations(rank_workload(w, rank), dev)
-    layer = MoeLayer(shape, wr, bias, w1, w3, w2, device=local_rank)
-    ctx = layer.ctx
-
-    # the workload's stand-in for the predictor: computed once, outside the timed region, with the
-    # library's own route + histogram (the prediction is an INPUT of the path)
-    ctx.route(x, wr, bias, layer.topk_idx, layer.topk_w)
-    ctx.histogram(layer.topk_idx, layer.hist)
-    true_hist = layer.hist.cpu()
-    if w.prediction == "true":
-        pred = true_hist.clone()
-    elif w.prediction == "noisy":
-        pred = wl.noisy_prediction(w, true_hist)
-    else:
-        xprev = wl.activations(w, dev, previous=True)
-        ctx.route(xprev, wr, bias, layer.topk_idx, layer.topk_w)
-        ctx.histogram(layer.topk_idx, layer.hist)
-        pred = layer.hist.cpu().clone()
-    pred_dev = pred.to(dev, torch.int32)
-
-    stream = torch.cuda.current_stream()
-    ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
-    gemm_marks = []
-
-    def step(record: bool):
-        ctx.plan(pred_dev, w.S, layer.replicas, layer.slot_off, layer.slot_expert, layer.bound)
-        ctx.route_histogram(x, wr, bias, layer.topk_idx, layer.topk_w, layer.hist)   # route + histogram fused
-        ctx.dispatch(x, layer.topk_idx, layer.hist, layer.replicas, layer.slot_off, layer.slot_row_off,
-                     layer.row_pair, layer.pair_row, layer.xp, layer.workspace)
-        if record:
-            a, b, c = ev(), ev(), ev()
-            a.record(stream)
-        ctx.expert_ffn_gate_up(layer.xp, layer.slot_row_off, layer.slot_expert, w1, w3, layer.h_ws)
-        if record:
-            b.record(stream)
-        ctx.expert_ffn_down(layer.h_ws, layer.slot_row_off, layer.slot_expert, w2, layer.yp)
-        if record:
-            c.record(stream)
-            gemm_marks.append((a, b, c))
-        ctx.combine(layer.yp, layer.pair_row, layer.topk_w, layer.out)
-
     def barrier():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
-        step(False)
-    barrier()
-    ctx.check_status()
-
+    w = wl.WORKLOADS[args.workload]
+    b = Bench(w, rank, local_rank)
     sampler = ClockSampler(visible_gpu_index(local_rank))
+    for _ in range(args.warmup):            # warm-up before the clock sampler starts, too
+        b.step(False)
+    barrier()
     if rank == 0:
         sampler.start()
         time.sleep(0.25)
-    launches0 = ctx.launch_count()
-    barrier()
-    t0, t1 = ev(), ev()
-    t0.record(stream)
-    for _ in range(args.steps):
-        step(True)
-    t1.record(stream)
-    barrier()
-    elapsed_ms = t0.elapsed_time(t1)
-    launches = ctx.launch_count() - launches0
+    elapsed_ms, gate_up_ms, down_ms, launches = b.timed_steps(args.steps, 0, barrier)
     clocks = sampler.stop() if rank == 0 else None
-    ctx.check_status()
     elapsed_ms = max_over_ranks(elapsed_ms, dist, dev)
     value = whole_job_rate(world, w.T, args.steps, elapsed_ms)
-
-    gate_up_ms = statistics.mean(a.elapsed_time(b) for a, b, _ in gemm_marks)
-    down_ms = statistics.mean(b.elapsed_time(c) for _, b, c in gemm_marks)
-
-    # end to end through the public layer API with host buffers (pinned), copies inside the timing
-    # (every step copies its batch in and its result out; HostPipeline overlaps the copies of
-    # neighbouring steps with the compute, as a serving loop would)
-    from paper_2506_07366_b200.layer import HostPipeline
-    xh = [x.cpu().pin_memory() for _ in range(2)]
-    oh = [torch.empty(w.T, w.D, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
-    pipe = HostPipeline(layer, depth=2)
-    layer.plan(pred_dev)
-    for i in range(max(2, min(3, args.warmup))):
-        pipe.submit(xh[i % 2], oh[i % 2])
-    pipe.drain()
-    barrier()
-    e0, e1 = ev(), ev()
-    e0.record(stream)
-    for i in range(args.steps):
-        layer.plan(pred_dev)
-        pipe.submit(xh[i % 2], oh[i % 2])
-    pipe.drain()
-    e1.record(stream)
-    barrier()
-    e2e_ms = e0.elapsed_time(e1)
-    e2e_ms = max_over_ranks(e2e_ms, dist, dev)
-    ctx.check_status()
+    e2e_ms = max_over_ranks(b.e2e_steps(args.steps, args.warmup, barrier), dist, dev)
     e2e_value = whole_job_rate(world, w.T, args.steps, e2e_ms)
 
     if rank != 0:
@@ -258,41 +456,27 @@ def run_ours(args):
         return
 
     peaks = measured_peaks()
-    kernels = per_call_timings(ctx, layer, w, x, wr, bias, w1, w3, w2, pred_dev, peaks) if world == 1 else None
-    flops_gate_up = 4.0 * w.R * w.D * w.F          # two of the three SwiGLU GEMMs, 2*R*D*F each
-    achieved = flops_gate_up / (gate_up_ms * 1e-3) / 1e12
-    ffn_tflops = 6.0 * w.R * w.D * w.F / ((gate_up_ms + down_ms) * 1e-3) / 1e12
-    hist_np = true_hist.numpy().astype("float64")
-    active = int((hist_np > 0).sum())
-    # slot loads of the last step: rows that carry a pair, counted per slot
-    occupied = (layer.row_pair >= 0).to(torch.int64).cumsum(0)
-    ends = layer.slot_row_off[1:].long().clamp(max=shape.Rcap) - 1
-    starts = layer.slot_row_off[:-1].long() - 1
-    cum_at = lambda i: torch.where(i >= 0, occupied[i.clamp(min=0)], torch.zeros_like(i))  # noqa: E731
-    slot_loads = (cum_at(ends) - cum_at(starts)).cpu().numpy()
-    err_dev = torch.zeros(1, dtype=torch.float64, device=dev)
-    ctx.error_rate(pred_dev, layer.hist, err_dev)
+    stats = b.load_statistics()
+    calls = b.per_call_timings(peaks) if world == 1 else None
+    ffn = b.ffn_summary(gate_up_ms, down_ms, peaks, stats["active_experts"])
+    achieved = 4.0 * w.R * w.D * w.F / (gate_up_ms * 1e-3) / 1e12      # two of the three SwiGLU GEMMs, 2*R*D*F each
     # a timed region of a few hundred ms runs at boost clocks: the burst peak is the fair denominator;
     # from a couple of seconds on, the power cap has settled and the sustained peak applies
     if elapsed_ms >= 2000.0:
         peak, peak_kind = peaks["bf16_sustained"], " (sustained bf16 GEMM: timed region >= 2 s)"
     else:
         peak, peak_kind = peaks["bf16_burst"], " (burst bf16 GEMM: timed region < 2 s, boost clocks)"
+    config = {"workload": w.name, "T": w.T, "D": w.D, "F": w.F, "E": w.E, "K": w.K, "S": w.S,
+              "row_align": Bench.A, "tokens_per_gpu": w.T, "prediction": w.prediction,
+              "l2": "inputs larger than L2: %.2f GB of expert weights stream through it every step"
+                    % (3 * w.E * w.D * w.F * 2 / 1e9)}
+    config.update({k: stats[k] for k in ("skewness", "skewness_after_plan", "max_slot_load", "plan_bound",
+                                         "prediction_error_rate", "max_replicas")})
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": w.name, "T": w.T, "D": w.D, "F": w.F, "E": w.E, "K": w.K, "S": w.S,
-                   "row_align": A, "tokens_per_gpu": w.T, "prediction": w.prediction,
-                   "skewness": float(hist_np.max() / (hist_np.sum() / w.E)),
-                   # the paper's load statistics of this batch, from the library's own outputs: the
-                   # bottleneck slot's load over the even share after duplication, the planner's
-                   # predicted bound, and the error rate of the prediction that drove the plan
-                   "skewness_after_plan": float(slot_loads.max() / (w.R / w.S)),
-                   "max_slot_load": int(slot_loads.max()), "plan_bound": int(layer.bound.item()),
-                   "prediction_error_rate": float(err_dev.item()),
-                   "l2": "inputs larger than L2: %.2f GB of expert weights stream through it every step"
-                         % (3 * w.E * w.D * w.F * 2 / 1e9)},
+        "config": config,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": w.T * w.D * 2,
                 "d2h_bytes_per_step": w.T * w.D * 2, "ms_per_step": e2e_ms / args.steps},
         "gpu_launches": int(launches),
@@ -302,114 +486,89 @@ def run_ours(args):
                      "frac_of_burst_peak": achieved / peaks["bf16_burst"],
                      "frac_of_sustained_peak": achieved / peaks["bf16_sustained"],
                      "peak_source": peaks["source"] + peak_kind,
-                     "ms_per_launch": gate_up_ms, "traffic": GATE_UP_DRAM_TRAFFIC.get(w.name)},
-        "expert_ffn": {"tflops": ffn_tflops, "gate_up_ms": gate_up_ms, "down_ms": down_ms,
-                       "frac_of_sustained_peak": ffn_tflops / peaks["bf16_sustained"],
-                       # the other roof of the grouped GEMMs: every expert that received tokens has its
-                       # weights streamed from HBM once per GEMM (binding when slots hold few rows)
-                       "active_experts": active,
-                       "gate_up_weight_gbs": active * 2.0 * w.D * w.F * 2 / (gate_up_ms * 1e-3) / 1e9,
-                       "down_weight_gbs": active * 1.0 * w.D * w.F * 2 / (down_ms * 1e-3) / 1e9,
-                       "gate_up_weight_frac_of_hbm_peak":
-                           active * 2.0 * w.D * w.F * 2 / (gate_up_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+                     "ms_per_launch": gate_up_ms, "traffic": recorded_traffic(w.name, w.R)},
+        "expert_ffn": ffn,
     }
-    if kernels is not None:
-        line["calls_cold_l2"] = kernels
+    if calls is not None:
+        line["calls_cold_l2"] = calls
     if world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_baseline(w, x, wr, bias, w1, w3, w2, pred)
+        line["cpu_baseline"] = cpu_baseline(w, b.x, b.wr, b.bias, b.w1, b.w3, b.w2, b.pred)
+    if world == 1 and not args.no_per_workload:
+        per = {}
+        b.close()
+        del b
+        for name in OTHER_WORKLOADS:
+            if name == w.name:
+                continue
+            torch.cuda.empty_cache()
+            ob = Bench(wl.WORKLOADS[name], 0, local_rank)
+            per[name] = compact_record(ob, peaks, args.per_workload_steps, barrier)
+            ob.close()
+            del ob
+        line["per_workload"] = per
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
 
 
-def per_call_timings(ctx, layer, w, x, wr, bias, w1, w3, w2, pred_dev, peaks, iters=7):
-    """Each library call timed alone (CUDA events on the launching stream, median of `iters`) with L2
-    flushed before every call by overwriting a 512 MB buffer, against the call's algorithmic HBM bytes
-    or flops.  The interval between the two events also holds the stream's launch gaps and the event
-    records themselves (`event_pair` = the same measurement with nothing in between), which matters
-    for calls of a few microseconds; kernel-only durations are in the ncu launch lists.  These
-    numbers explain the step time; they are not part of the timed step."""
-    stream = torch.cuda.current_stream()
-    flush = torch.empty(512 << 20, dtype=torch.uint8, device=x.device)
-    R, T, D, F, E, K = w.R, w.T, w.D, w.F, w.E, w.K
-    ctx.plan(pred_dev, w.S, layer.replicas, layer.slot_off, layer.slot_expert, layer.bound)
-    calls = [
-        ("plan", lambda: ctx.plan(pred_dev, w.S, layer.replicas, layer.slot_off, layer.slot_expert, layer.bound),
-         None, None),
-        ("route", lambda: ctx.route(x, wr, bias, layer.topk_idx, layer.topk_w),
-         2.0 * T * D + 2.0 * E * D + 8.0 * T * K, 2.0 * T * D * E),
-        ("histogram", lambda: ctx.histogram(layer.topk_idx, layer.hist), 4.0 * R, None),
-        ("route_histogram", lambda: ctx.route_histogram(x, wr, bias, layer.topk_idx, layer.topk_w, layer.hist),
-         2.0 * T * D + 2.0 * E * D + 8.0 * T * K, 2.0 * T * D * E),
-        ("dispatch", lambda: ctx.dispatch(x, layer.topk_idx, layer.hist, layer.replicas, layer.slot_off,
-                                          layer.slot_row_off, layer.row_pair, layer.pair_row, layer.xp,
-                                          layer.workspace), 2.0 * T * D + 2.0 * R * D + 12.0 * R, None),
-        ("expert_ffn_gate_up", lambda: ctx.expert_ffn_gate_up(layer.xp, layer.slot_row_off, layer.slot_expert, w1, w3,
-                                                              layer.h_ws), None, 4.0 * R * D * F),
-        ("expert_ffn_down", lambda: ctx.expert_ffn_down(layer.h_ws, layer.slot_row_off, layer.slot_expert, w2,
-                                                        layer.yp), None, 2.0 * R * D * F),
-        ("combine", lambda: ctx.combine(layer.yp, layer.pair_row, layer.topk_w, layer.out),
-         2.0 * R * D + 2.0 * T * D + 8.0 * R, None),
-    ]
-    out = {}
-    calls.append(("event_pair", lambda: None, None, None))
-    for name, fn, nbytes, flops in calls:
-        times = []
-        for _ in range(iters):
-            flush.fill_(1)
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            fn()
-            b.record(stream)
-            b.synchronize()
-            times.append(a.elapsed_time(b))
-        ms = statistics.median(times)
-        rec = {"us": ms * 1e3}
-        if nbytes is not None:
-            rec["gbs"] = nbytes / (ms * 1e-3) / 1e9
-            rec["frac_of_hbm_peak"] = rec["gbs"] / peaks["hbm_gbs"]
-        if flops is not None and name.startswith("expert"):
-            rec["tflops"] = flops / (ms * 1e-3) / 1e12
-            rec["frac_of_burst_peak"] = rec["tflops"] / peaks["bf16_burst"]
-        out[name] = rec
-    ctx.check_status()
-    return out
-
-
 # ------------------------------------------------------------------------------------- oracle arm
-def oracle_sample_step(w, xb, wrb, bias, w1, w3, w2, pred, n_tokens):
-    """One pass of the oracle over the first n_tokens tokens of the batch."""
-    import oracle
-    sub = xb[:n_tokens]
-    return oracle.moe_layer(sub, wrb, bias, w1, w3, w2, pred, K=w.K, S=w.S, gate_mode=w.gate_mode, row_align=1)
-
-
 class _HostExperts:
+    """w[e] -> host bf16 bits of one expert's matrix, fetched from the device on first use."""
+
     def __init__(self, t):
-        self.t = t
-        self.shape = tuple(t.shape)
+        self.t, self.shape, self.cache = t, tuple(t.shape), {}
 
     def __getitem__(self, e):
-        return wl.bf16_bits(self.t[int(e)])
+        e = int(e)
+        if e not in self.cache:
+            self.cache[e] = wl.bf16_bits(self.t[e])
+        return self.cache[e]
 
 
-def cpu_baseline(w, x, wr, bias, w1, w3, w2, pred, n_tokens=None, seconds_hint=120.0):
-    """Times the oracle, as it stands, on the host cores over a bounded sample of the workload."""
-    import numpy as np
+def oracle_sample_tokens(w) -> int:
+    """Tokens per oracle pass: sized so that one pass takes a few seconds on the host cores (the
+    cost is about 6*D*F fp64 multiply-adds per routed pair plus decoding every used expert's weights)."""
+    per_token = 6.0 * w.K * w.D * w.F
+    return int(max(8, min(w.T, 50.0 * 2e10 / per_token)))
+
+
+class OracleSample:
+    """The first n tokens of a workload's batch with everything the oracle needs on the host."""
+
+    def __init__(self, w, x, wr, bias, w1, w3, w2, pred):
+        import numpy as np
+        self.w, self.n = w, oracle_sample_tokens(w)
+        self.xb, self.wrb, self.b = wl.bf16_bits(x[:self.n]), wl.bf16_bits(wr), bias.cpu().numpy()
+        self.experts = [_HostExperts(t) for t in (w1, w3, w2)]
+        self.pred = np.asarray(pred)
+
+    def one_pass(self) -> float:
+        """One pass of the oracle, as it stands, over the sample; returns the seconds it took."""
+        import oracle
+        w = self.w
+        t0 = time.perf_counter()
+        oracle.moe_layer(self.xb, self.wrb, self.b, *self.experts, self.pred, K=w.K, S=w.S, gate_mode=w.gate_mode,
+                         row_align=1)
+        return time.perf_counter() - t0
+
+    def describe(self) -> str:
+        return (f"first {self.n} of {self.w.T} tokens of '{self.w.name}', all experts' weights (bf16 bits on the "
+                f"host, fetched before the timing; decoding them to fp64 is part of every pass)")
+
+
+def host_threads() -> int:
     from threadpoolctl import threadpool_info
-    # the oracle's cost is dominated by 6*D*F MACs per routed pair at a few GFLOP/s per core
-    if n_tokens is None:
-        per_token = 6.0 * w.K * w.D * w.F
-        n_tokens = int(max(8, min(w.T, seconds_hint * 2e10 / per_token)))
-    xb, wrb, b = wl.bf16_bits(x[:n_tokens]), wl.bf16_bits(wr), bias.cpu().numpy()
-    ex1, ex3, ex2 = _HostExperts(w1), _HostExperts(w3), _HostExperts(w2)
-    t0 = time.perf_counter()
-    oracle_sample_step(w, xb, wrb, b, ex1, ex3, ex2, np.asarray(pred), n_tokens)
-    dt = time.perf_counter() - t0
-    threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
-    return {"value": n_tokens / dt, "unit": UNIT, "cores": int(threads), "kind": "oracle",
-            "sample": f"first {n_tokens} of {w.T} tokens of '{w.name}', all experts' weights, one pass "
-                      f"(includes fetching each used expert's weights to the host), {dt:.1f} s"}
+    return int(max([p.get("num_threads", 1) for p in threadpool_info()] + [1]))
+
+
+def cpu_baseline(w, x, wr, bias, w1, w3, w2, pred, passes=2):
+    """Times the oracle, as it stands, on the host cores over a bounded sample of the workload: one
+    untimed pass (it also brings the weights to the host), then `passes` timed ones."""
+    s = OracleSample(w, x, wr, bias, w1, w3, w2, pred)
+    s.one_pass()
+    dt = sum(s.one_pass() for _ in range(passes))
+    return {"value": s.n * passes / dt, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
+            "sample": f"{s.describe()}; {passes} passes, {dt / passes:.1f} s each"}
 
 
 def run_reference(args):
@@ -423,21 +582,18 @@ def run_reference(args):
     w1, w3, w2 = wl.expert_weights(w, dev)
     x = wl.activations(w, dev)
     pred = np.full(w.E, w.R // w.E, dtype=np.int64)
-    per_token = 6.0 * w.K * w.D * w.F
-    n_tokens = int(max(8, min(w.T, 6.0 * 2e10 / per_token)))
-    times = []
-    for i in range(args.warmup + args.steps):
-        r = cpu_baseline(w, x, wr, bias, w1, w3, w2, pred, n_tokens=n_tokens)
-        if i >= args.warmup:
-            times.append(n_tokens / r["value"])
+    s = OracleSample(w, x, wr, bias, w1, w3, w2, pred)          # the same sample as the cpu_baseline leg
+    for _ in range(max(1, args.warmup)):
+        s.one_pass()
+    times = [s.one_pass() for _ in range(args.steps)]
     dt = sum(times)
-    value = n_tokens * len(times) / dt
+    value = s.n * len(times) / dt
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / len(times) * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": w.name, "T": w.T, "D": w.D, "F": w.F, "E": w.E, "K": w.K, "S": w.S},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": r["cores"], "kind": "oracle",
-                             "sample": f"each step = first {n_tokens} of {w.T} tokens, all experts' weights"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
+                             "sample": f"each step = {s.describe()}"},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
@@ -448,10 +604,21 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="mixtral", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(wl.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-workload", action="store_true",
+                    help="skip the short measurements of the other full-size workloads")
+    ap.add_argument("--per-workload-steps", type=int, default=10)
+    ap.add_argument("--record-traffic", metavar="NCU_CSV",
+                    help="store the grouped GEMMs' DRAM byte counters of an ncu --csv log (taken on "
+                         "--workload, --traffic-pairs routed pairs per launch) in profiles/dram_traffic.json")
+    ap.add_argument("--traffic-pairs", type=int, default=0)
     args = ap.parse_args()
+    if args.record_traffic:
+        w = wl.WORKLOADS[args.workload]
+        record_traffic(args.record_traffic, w.name, args.traffic_pairs or w.R)
+        return
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":

@@ -26,6 +26,11 @@
  *    host before anything is launched; a failing call launches nothing.  Conditions only the device
  *    can see (an expert index out of range, a wait that ran out) are recorded in a device status
  *    word that moegps_status reads; the kernels skip the offending access instead of faulting.
+ *  - A context belongs to the device it was created on, and that device must be the calling
+ *    thread's current device in every call that launches work (and in moegps_status); otherwise the
+ *    call returns MOEGPS_ERR_INVALID_ARG and launches nothing.
+ *  - Device-side index checks: a slot extent, row or expert index outside its range is skipped (no
+ *    out-of-range read or write is made for it) and MOEGPS_ERR_BAD_INDEX is recorded.
  *  - Weight layouts are "output features x input features", so both GEMM operands are contiguous
  *    along the contraction.
  */
@@ -49,7 +54,8 @@ typedef enum moegps_error {
   MOEGPS_OK = 0,
   MOEGPS_ERR_INVALID_ARG = -1,         /* null or misaligned pointer, n_slots != S, bad enum value   */
   MOEGPS_ERR_UNSUPPORTED_SHAPE = -2,   /* a dimension outside the limits listed at moegps_shape_t    */
-  MOEGPS_ERR_WORKSPACE_TOO_SMALL = -3,
+  MOEGPS_ERR_WORKSPACE_TOO_SMALL = -3, /* raised only by a binding that knows the buffer's size: the C calls
+                                          take a bare pointer and cannot check it (see moegps_dispatch)  */
   MOEGPS_ERR_CUDA = -4,                /* a CUDA runtime/driver call failed (see moegps_last_cuda_error) */
   MOEGPS_ERR_UNIMPLEMENTED = -5,
   MOEGPS_ERR_BAD_INDEX = -6,           /* device: an expert/row index outside its range was skipped  */
@@ -129,7 +135,9 @@ MOEGPS_API int moegps_plan(moegps_ctx_t* ctx, const int32_t* predicted_hist, int
  * slot_row_off: int32 [S+1], slot s owns rows slot_row_off[s]..slot_row_off[s+1]-1, starts are
  *   multiples of row_align; row_pair: int32 [Rcap] (flat pair of each occupied row, -1 on padding);
  * pair_row: int32 [T,K]; xp: bf16 [Rcap,D] (padding rows are not written).
- * workspace: moegps_workspace_bytes(shape) bytes of scratch, contents irrelevant. */
+ * workspace: moegps_workspace_bytes(shape) bytes of scratch, contents irrelevant.  Its size cannot be
+ *   checked here (only a pointer is passed): a buffer shorter than that is the caller's error.
+ *   Calls that may overlap on the GPU need a workspace each. */
 MOEGPS_API int moegps_dispatch(moegps_ctx_t* ctx, const void* x, const int32_t* topk_idx, const int32_t* hist,
                     const int32_t* replicas, const int32_t* slot_off,
                     int32_t* slot_row_off, int32_t* row_pair, int32_t* pair_row,
@@ -170,7 +178,9 @@ MOEGPS_API int moegps_dispatch_static(moegps_ctx_t* ctx, const void* x, const in
  * xp: bf16 [Rcap,D]; slot_row_off: int32 [S+1]; slot_expert: int32 [S];
  * w_gate, w_up: bf16 [E,F,D]; w_down: bf16 [E,D,F]; h_ws: bf16 [Rcap,F] scratch; yp: bf16 [Rcap,D].
  * All rows of a slot's extent are computed (padding rows yield unspecified values); rows outside
- * every slot and slots with slot_expert < 0 are not written. */
+ * every slot and slots with slot_expert < 0 are not written.  A slot whose extent in slot_row_off
+ * is not inside [0, Rcap] (negative, decreasing, or past the buffers) is skipped entirely and
+ * MOEGPS_ERR_BAD_INDEX is recorded. */
 MOEGPS_API int moegps_expert_ffn(moegps_ctx_t* ctx, const void* xp, const int32_t* slot_row_off,
                       const int32_t* slot_expert, const void* w_gate, const void* w_up,
                       const void* w_down, void* h_ws, void* yp, void* stream);
@@ -192,8 +202,7 @@ MOEGPS_API int moegps_combine(moegps_ctx_t* ctx, const void* yp, const int32_t* 
                    void* out, void* stream);
 
 /* predictor_update - state of Distribution-Only Prediction across batches (paper, Section 3.2.1:
- * the maximum-likelihood estimate p_e = n_e / N of Eq. 1, which becomes a moving average when the
- * data arrive as batches).  state[e] += hist[e]; state / sum(state) is then Eq. 1 over all tokens
+ * the maximum-likelihood estimate p_e = n_e / N of Eq. 1, averaged over the batches seen).  state[e] += hist[e]; state / sum(state) is then Eq. 1 over all tokens
  * seen.  predicted_hist = state divided by the smallest power of two that makes its largest entry fit
  * an int32 (the planner only uses proportions) - ready to be passed to moegps_plan for the next
  * batch.  hist: int32 [E] >= 0; state: int64 [E], zeroed by the caller to start or restart;

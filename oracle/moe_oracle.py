@@ -126,8 +126,8 @@ def skewness(hist) -> float:
 
 
 def error_rate(p_est, p_true) -> float:
-    """|p_est - p_true| measured in units of 1/E and averaged over the experts (Section 3.2.1 with
-    the "averaged L1 distance over number of experts" of Section 3.3)."""
+    """|p_est - p_true| measured in units of 1/E (Section 3.2.1), averaged over the experts as
+    Section 3.3 reads it."""
     a = np.asarray(p_est, dtype=np.float64)
     b = np.asarray(p_true, dtype=np.float64)
     E = a.size
@@ -135,8 +135,8 @@ def error_rate(p_est, p_true) -> float:
 
 
 def predictor_update(state, hist):
-    """Distribution-Only predictor state over batches (Section 3.2.1: with batched data the
-    estimate of Eq. 1 becomes a moving average): the state holds the per-expert counts of all
+    """Distribution-Only predictor state over batches (Section 3.2.1, the estimate of Eq. 1
+    averaged over the batches seen): the state holds the per-expert counts of all
     batches seen, so state / sum(state) is the maximum-likelihood estimate over the pooled tokens.
     Returns (new_state as Python ints, predicted_hist int32): the prediction handed to the planner
     is the state itself, divided by the smallest power of two that makes its largest entry fit an

@@ -83,13 +83,15 @@ size_t moegps_workspace_bytes(const moegps_shape_t* shape) {
   if (check_shape(shape) != MOEGPS_OK) return 0;
   const int64_t R = (int64_t)shape->T * shape->K;
   const int64_t nseg = (R + kSegPairs - 1) / kSegPairs;
-  size_t bytes = (size_t)(nseg > 0 ? nseg : 1) * shape->E * sizeof(int32_t);
+  // the per-(segment, expert) count matrix + one word for the scan path's ticket counter
+  size_t bytes = ((size_t)(nseg > 0 ? nseg : 1) * shape->E + 1) * sizeof(int32_t);
   return (bytes + 255) & ~(size_t)255;
 }
 
 int moegps_route(moegps_ctx_t* ctx, const void* x, const void* w_router, const float* bias,
                  int32_t* topk_idx, float* topk_w, void* stream) {
   if (!ctx) return MOEGPS_ERR_INVALID_ARG;
+  if (int rc = moegps_check_device(ctx)) return rc;
   if (ctx->shape.T == 0) return MOEGPS_OK;          // nothing to route (empty tensors have no address)
   if (!all_ok(x, w_router, topk_idx, topk_w)) return MOEGPS_ERR_INVALID_ARG;
   if (bias && (reinterpret_cast<uintptr_t>(bias) & 3u)) return MOEGPS_ERR_INVALID_ARG;
@@ -99,6 +101,7 @@ int moegps_route(moegps_ctx_t* ctx, const void* x, const void* w_router, const f
 int moegps_route_histogram(moegps_ctx_t* ctx, const void* x, const void* w_router, const float* bias,
                            int32_t* topk_idx, float* topk_w, int32_t* hist, void* stream) {
   if (!ctx || !all_ok(hist)) return MOEGPS_ERR_INVALID_ARG;
+  if (int rc = moegps_check_device(ctx)) return rc;
   if (ctx->shape.T == 0)                            // no tokens: the histogram is all zero
     return cudaMemsetAsync(hist, 0, sizeof(int32_t) * ctx->shape.E, (cudaStream_t)stream) == cudaSuccess
                ? MOEGPS_OK : MOEGPS_ERR_CUDA;
@@ -110,6 +113,7 @@ int moegps_route_histogram(moegps_ctx_t* ctx, const void* x, const void* w_route
 int moegps_route_logits(moegps_ctx_t* ctx, const void* x, const void* w_router, const float* bias,
                         float* logits, void* stream) {
   if (!ctx) return MOEGPS_ERR_INVALID_ARG;
+  if (int rc = moegps_check_device(ctx)) return rc;
   if (ctx->shape.T == 0) return MOEGPS_OK;
   if (!all_ok(x, w_router, logits)) return MOEGPS_ERR_INVALID_ARG;
   if (bias && (reinterpret_cast<uintptr_t>(bias) & 3u)) return MOEGPS_ERR_INVALID_ARG;
@@ -118,6 +122,7 @@ int moegps_route_logits(moegps_ctx_t* ctx, const void* x, const void* w_router, 
 
 int moegps_histogram(moegps_ctx_t* ctx, const int32_t* topk_idx, int32_t* hist, void* stream) {
   if (!ctx || !all_ok(hist)) return MOEGPS_ERR_INVALID_ARG;
+  if (int rc = moegps_check_device(ctx)) return rc;
   if (ctx->shape.T > 0 && !all_ok(topk_idx)) return MOEGPS_ERR_INVALID_ARG;
   return moegps_launch_histogram(ctx, topk_idx, hist, (cudaStream_t)stream);
 }
@@ -125,6 +130,7 @@ int moegps_histogram(moegps_ctx_t* ctx, const int32_t* topk_idx, int32_t* hist, 
 int moegps_plan(moegps_ctx_t* ctx, const int32_t* predicted_hist, int32_t n_slots, int32_t* replicas,
                 int32_t* slot_off, int32_t* slot_expert, int32_t* bound, void* stream) {
   if (!ctx || !all_ok(predicted_hist, replicas, slot_off, slot_expert) || !bound) return MOEGPS_ERR_INVALID_ARG;
+  if (int rc = moegps_check_device(ctx)) return rc;
   if (reinterpret_cast<uintptr_t>(bound) & 3u) return MOEGPS_ERR_INVALID_ARG;
   if (n_slots != ctx->shape.S) return MOEGPS_ERR_INVALID_ARG;
   return moegps_launch_plan(ctx, predicted_hist, replicas, slot_off, slot_expert, bound, (cudaStream_t)stream);
@@ -134,6 +140,7 @@ int moegps_dispatch(moegps_ctx_t* ctx, const void* x, const int32_t* topk_idx, c
                     const int32_t* replicas, const int32_t* slot_off, int32_t* slot_row_off,
                     int32_t* row_pair, int32_t* pair_row, void* xp, void* workspace, void* stream) {
   if (!ctx || !all_ok(hist, replicas, slot_off, slot_row_off, workspace)) return MOEGPS_ERR_INVALID_ARG;
+  if (int rc = moegps_check_device(ctx)) return rc;
   if (ctx->shape.T > 0 && !all_ok(x, topk_idx, pair_row, xp)) return MOEGPS_ERR_INVALID_ARG;
   if (moegps_rcap_of(ctx->shape) > 0 && !all_ok(row_pair)) return MOEGPS_ERR_INVALID_ARG;
   return moegps_launch_dispatch(ctx, x, topk_idx, hist, replicas, slot_off, slot_row_off, row_pair, pair_row,
@@ -144,6 +151,7 @@ int moegps_expert_ffn(moegps_ctx_t* ctx, const void* xp, const int32_t* slot_row
                       const int32_t* slot_expert, const void* w_gate, const void* w_up, const void* w_down,
                       void* h_ws, void* yp, void* stream) {
   if (!ctx) return MOEGPS_ERR_INVALID_ARG;
+  if (int rc = moegps_check_device(ctx)) return rc;
   if (ctx->shape.T == 0) return MOEGPS_OK;
   if (!all_ok(xp, slot_row_off, slot_expert, w_gate, w_up, w_down, h_ws, yp)) return MOEGPS_ERR_INVALID_ARG;
   int rc = moegps_launch_ffn_gate_up(ctx, xp, slot_row_off, slot_expert, w_gate, w_up, h_ws, (cudaStream_t)stream);
@@ -155,6 +163,7 @@ int moegps_expert_ffn_gate_up(moegps_ctx_t* ctx, const void* xp, const int32_t* 
                               const int32_t* slot_expert, const void* w_gate, const void* w_up, void* h_ws,
                               void* stream) {
   if (!ctx) return MOEGPS_ERR_INVALID_ARG;
+  if (int rc = moegps_check_device(ctx)) return rc;
   if (ctx->shape.T == 0) return MOEGPS_OK;
   if (!all_ok(xp, slot_row_off, slot_expert, w_gate, w_up, h_ws)) return MOEGPS_ERR_INVALID_ARG;
   return moegps_launch_ffn_gate_up(ctx, xp, slot_row_off, slot_expert, w_gate, w_up, h_ws, (cudaStream_t)stream);
@@ -163,6 +172,7 @@ int moegps_expert_ffn_gate_up(moegps_ctx_t* ctx, const void* xp, const int32_t* 
 int moegps_expert_ffn_down(moegps_ctx_t* ctx, const void* h_ws, const int32_t* slot_row_off,
                            const int32_t* slot_expert, const void* w_down, void* yp, void* stream) {
   if (!ctx) return MOEGPS_ERR_INVALID_ARG;
+  if (int rc = moegps_check_device(ctx)) return rc;
   if (ctx->shape.T == 0) return MOEGPS_OK;
   if (!all_ok(h_ws, slot_row_off, slot_expert, w_down, yp)) return MOEGPS_ERR_INVALID_ARG;
   return moegps_launch_ffn_down(ctx, h_ws, slot_row_off, slot_expert, w_down, yp, (cudaStream_t)stream);
@@ -171,6 +181,7 @@ int moegps_expert_ffn_down(moegps_ctx_t* ctx, const void* h_ws, const int32_t* s
 int moegps_combine(moegps_ctx_t* ctx, const void* yp, const int32_t* pair_row, const float* topk_w,
                    void* out, void* stream) {
   if (!ctx) return MOEGPS_ERR_INVALID_ARG;
+  if (int rc = moegps_check_device(ctx)) return rc;
   if (ctx->shape.T == 0) return MOEGPS_OK;
   if (!all_ok(yp, pair_row, topk_w, out)) return MOEGPS_ERR_INVALID_ARG;
   return moegps_launch_combine(ctx, yp, pair_row, topk_w, out, (cudaStream_t)stream);
@@ -178,8 +189,9 @@ int moegps_combine(moegps_ctx_t* ctx, const void* yp, const int32_t* pair_row, c
 
 int moegps_status(moegps_ctx_t* ctx, void* stream, int32_t* host_status) {
   if (!ctx || !host_status) return MOEGPS_ERR_INVALID_ARG;
+  if (int rc = moegps_check_device(ctx)) return rc;
   cudaStream_t st = (cudaStream_t)stream;
-  int32_t h[4] = {0, 0, 0, 0};
+  int32_t h[2] = {0, 0};      // error code and its detail
   MOEGPS_CUDA_TRY(ctx, cudaMemcpyAsync(h, ctx->d_status, sizeof(h), cudaMemcpyDeviceToHost, st));
   MOEGPS_CUDA_TRY(ctx, cudaMemsetAsync(ctx->d_status, 0, sizeof(h), st));
   MOEGPS_CUDA_TRY(ctx, cudaStreamSynchronize(st));

@@ -8,7 +8,7 @@
 
 #include "moegps.h"
 
-// Layout of the device status word: [0] first error code, [1] detail (index / location), [2..3] spare.
+// Layout of the device status word: [0] first error code, [1] detail (index / location), [2..3] unused.
 struct moegps_ctx {
   moegps_shape_t shape;
   int device;
@@ -56,6 +56,14 @@ static inline bool moegps_aligned16(const void* p) { return (reinterpret_cast<ui
 
 static inline int64_t moegps_rcap_of(const moegps_shape_t& s) {
   return (int64_t)s.T * s.K + (int64_t)s.S * (s.row_align - 1);
+}
+
+// The status word, the cached tensor maps and the kernel attributes of a context belong to its
+// device, so that device must be the calling thread's current one; otherwise nothing is launched.
+static inline int moegps_check_device(const moegps_ctx* ctx) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return MOEGPS_ERR_CUDA;
+  return dev == ctx->device ? MOEGPS_OK : MOEGPS_ERR_INVALID_ARG;
 }
 
 // First error wins; later ones are dropped.

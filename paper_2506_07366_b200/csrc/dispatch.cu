@@ -7,8 +7,10 @@
 //                   workspace[e][seg], and CTA 0 also derives the slot row offsets from hist /
 //                   replicas / row_align (they do not depend on the counts) with a block scan.
 //                   Longer pair lists (count_scan): counts are stored workspace[seg][e] and the CTA
-//                   that finishes last (ticket counter, no waiting) turns them into per-expert
-//                   exclusive prefix sums over the segments before it derives the offsets.
+//                   that finishes last (a ticket counter kept in the call's own scratch, right behind
+//                   the count matrix and zeroed on the stream before the launch; no waiting) turns
+//                   them into per-expert exclusive prefix sums over the segments before it derives
+//                   the offsets.
 //   2. rank_copy  : one warp per token.  The stable rank of a pair is its segment's base plus the
 //                   number of earlier same-expert pairs inside the segment, which the warp counts
 //                   from the segment's indices (a 1 KiB read).  The base is read from the scanned
@@ -18,6 +20,8 @@
 //                   in integer arithmetic.  The warp then reads the token row once (128-bit loads)
 //                   and writes it to its K rows of the permuted buffer (128-bit stores).
 // Stable by construction, integer only, no atomics on results => bit-exact and deterministic.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace {
@@ -129,7 +133,7 @@ count_scan_kernel(const int32_t* __restrict__ topk_idx, int64_t R, int E, int S,
                   int32_t* seg_cnt, int nseg, int32_t* __restrict__ row_pair, int64_t Rcap,
                   const int32_t* __restrict__ hist, const int32_t* __restrict__ replicas,
                   const int32_t* __restrict__ slot_off, int32_t* __restrict__ slot_row_off,
-                  int e_chunk, int32_t* status) {
+                  int e_chunk, int32_t* __restrict__ ticket_ctr, int32_t* status) {
   __shared__ int32_t cnt[kMaxE];
   __shared__ int32_t padded[kMaxS];     // rows reserved for each slot (load rounded up to A)
   __shared__ int32_t warp_tot[32];
@@ -160,9 +164,8 @@ count_scan_kernel(const int32_t* __restrict__ topk_idx, int64_t R, int E, int S,
   __threadfence();
   __syncthreads();
   if (tid == 0) {
-    const int ticket = atomicAdd(&status[2], 1);
+    const int ticket = atomicAdd(ticket_ctr, 1);
     is_last = ticket == (int)gridDim.x - 1;
-    if (is_last) status[2] = 0;               // ready for the next call
   }
   __syncthreads();
   if (!is_last) return;
@@ -391,9 +394,11 @@ int moegps_launch_dispatch(moegps_ctx* ctx, const void* x, const int32_t* topk_i
     count_kernel<<<nseg > 0 ? nseg : 1, kSegPairs, 0, st>>>(topk_idx, R, s.E, s.S, s.row_align, seg, nseg, row_pair, Rcap,
                                                             hist, replicas, slot_off, slot_row_off, ctx->d_status);
   } else {
+    int32_t* ticket = seg + (int64_t)nseg * s.E;     // the scratch's last word (see moegps_workspace_bytes)
+    MOEGPS_CUDA_TRY(ctx, cudaMemsetAsync(ticket, 0, sizeof(int32_t), st));
     count_scan_kernel<<<nseg, kScanThreads, scan_smem, st>>>(topk_idx, R, s.E, s.S, s.row_align, seg, nseg, row_pair,
                                                              Rcap, hist, replicas, slot_off, slot_row_off, e_chunk,
-                                                             ctx->d_status);
+                                                             ticket, ctx->d_status);
   }
   MOEGPS_AFTER_LAUNCH(ctx);
   if (R == 0) return MOEGPS_OK;
@@ -420,10 +425,12 @@ int moegps_launch_dispatch(moegps_ctx* ctx, const void* x, const int32_t* topk_i
 namespace {
 
 constexpr size_t kStaticScratchInts = 262144;                    // 1 MiB of int32 counters
-static __device__ __align__(256) int32_t g_dispatch_scratch[kStaticScratchInts];
+// (+ 64: the word behind the largest count matrix is the scan path's ticket counter)
+static __device__ __align__(256) int32_t g_dispatch_scratch[kStaticScratchInts + 64];
 
 constexpr int kMaxDevices = 64;
-int32_t* g_scratch_addr[kMaxDevices] = {};                       // device address of the array, per device
+// device address of the array, per device; atomics because host threads may race to the first call
+std::atomic<int32_t*> g_scratch_addr[kMaxDevices];
 
 }  // namespace
 
@@ -446,17 +453,18 @@ extern "C" MOEGPS_API int moegps_dispatch_static(moegps_ctx_t* ctx, const void* 
   const int64_t R = (int64_t)s.T * s.K;
   const int64_t nseg = (R + kSegPairs - 1) / kSegPairs;
   if ((uint64_t)(nseg * s.E) > kStaticScratchInts) return MOEGPS_ERR_STATIC_SCRATCH_EXCEEDED;
-  int dev = -1;
-  MOEGPS_CUDA_TRY(ctx, cudaGetDevice(&dev));
-  if (dev != ctx->device || dev < 0 || dev >= kMaxDevices) return MOEGPS_ERR_INVALID_ARG;
-  if (!g_scratch_addr[dev]) {
+  if (int rc = moegps_check_device(ctx)) return rc;
+  const int dev = ctx->device;
+  if (dev < 0 || dev >= kMaxDevices) return MOEGPS_ERR_INVALID_ARG;
+  int32_t* scratch = g_scratch_addr[dev].load(std::memory_order_acquire);
+  if (!scratch) {
     // In host code the array's name is only a handle; the address a kernel can use has to be asked
-    // for, once per device, with that device current.
-    int32_t* p = nullptr;
-    MOEGPS_CUDA_TRY(ctx, cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_dispatch_scratch));
-    if (!p) return MOEGPS_ERR_CUDA;
-    g_scratch_addr[dev] = p;
+    // for, once per device, with that device current.  (Two threads racing here both get the same
+    // answer, so the second store is harmless.)
+    MOEGPS_CUDA_TRY(ctx, cudaGetSymbolAddress(reinterpret_cast<void**>(&scratch), g_dispatch_scratch));
+    if (!scratch) return MOEGPS_ERR_CUDA;
+    g_scratch_addr[dev].store(scratch, std::memory_order_release);
   }
   return moegps_launch_dispatch(ctx, x, topk_idx, hist, replicas, slot_off, slot_row_off, row_pair, pair_row, xp,
-                                g_scratch_addr[dev], (cudaStream_t)stream);
+                                scratch, (cudaStream_t)stream);
 }

@@ -144,7 +144,7 @@ template <bool kSwiGLU>
 __global__ void __launch_bounds__(kThreads, 1)
 grouped_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
                     const __grid_constant__ CUtensorMap tm_b1, const int32_t* __restrict__ slot_row_off,
-                    const int32_t* __restrict__ slot_expert, int S, int E, int n_dim, int k_dim,
+                    const int32_t* __restrict__ slot_expert, int S, int E, int n_dim, int k_dim, int rcap,
                     __nv_bfloat16* __restrict__ out, int32_t* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -185,10 +185,16 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     int acc = 0;
     for (int s = 0; s < S; ++s) {
       tb.tile_base[s] = acc;
-      const int rows = tb.row_off[s + 1] - tb.row_off[s];
+      // a slot whose extent is not inside [0, rcap] (offsets negative, decreasing or past the
+      // buffers) gets no tiles: nothing is read or written for it, and the caller is told
+      const int lo = tb.row_off[s], hi = tb.row_off[s + 1];
       const int e = tb.expert[s];
-      if (rows > 0 && e >= 0 && e < E) acc += ((rows + BM - 1) / BM) * n_tiles;
-      else if (rows > 0 && e >= E) moegps_report(status, MOEGPS_ERR_BAD_INDEX, s);
+      if (lo < 0 || hi < lo || hi > rcap) {
+        moegps_report(status, MOEGPS_ERR_BAD_INDEX, s);
+        continue;
+      }
+      if (hi > lo && e >= 0 && e < E) acc += ((hi - lo + BM - 1) / BM) * n_tiles;
+      else if (hi > lo && e >= E) moegps_report(status, MOEGPS_ERR_BAD_INDEX, s);
     }
     tb.tile_base[S] = acc;
     *total_tiles_p = acc;
@@ -379,7 +385,7 @@ int moegps_launch_ffn_gate_up(moegps_ctx* ctx, const void* xp, const int32_t* sl
   int rc = raise_smem_limit(ctx);
   if (rc != MOEGPS_OK) return rc;
   grouped_gemm_kernel<true><<<ctx->sm_count, kThreads, kSmemBytes, st>>>(
-      ctx->tm_xp, ctx->tm_w1, ctx->tm_w3, slot_row_off, slot_expert, s.S, s.E, s.F, s.D,
+      ctx->tm_xp, ctx->tm_w1, ctx->tm_w3, slot_row_off, slot_expert, s.S, s.E, s.F, s.D, (int)rcap,
       static_cast<__nv_bfloat16*>(h_ws), ctx->d_status);
   MOEGPS_AFTER_LAUNCH(ctx);
   return MOEGPS_OK;
@@ -400,7 +406,7 @@ int moegps_launch_ffn_down(moegps_ctx* ctx, const void* h_ws, const int32_t* slo
   int rc = raise_smem_limit(ctx);
   if (rc != MOEGPS_OK) return rc;
   grouped_gemm_kernel<false><<<ctx->sm_count, kThreads, kSmemBytes, st>>>(
-      ctx->tm_h, ctx->tm_w2, ctx->tm_w2, slot_row_off, slot_expert, s.S, s.E, s.D, s.F,
+      ctx->tm_h, ctx->tm_w2, ctx->tm_w2, slot_row_off, slot_expert, s.S, s.E, s.D, s.F, (int)rcap,
       static_cast<__nv_bfloat16*>(yp), ctx->d_status);
   MOEGPS_AFTER_LAUNCH(ctx);
   return MOEGPS_OK;

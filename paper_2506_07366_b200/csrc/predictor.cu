@@ -1,7 +1,8 @@
 // Distribution-Only Prediction state on the device (paper, Section 3.2.1): the maximum-likelihood
 // estimate p_e = n_e / N of Eq. 1 over all batches seen so far is kept as cumulative per-expert
-// counts ("when the data come as batches the estimation becomes a moving average"), and the error
-// rate |p_est - p| / (1/E), averaged over the experts, compares a prediction with what a batch did.
+// counts, i.e. Eq. 1 over the pooled tokens (the running average Section 3.2.1 describes for batched
+// data), and the error rate |p_est - p| / (1/E) of Section 3.2.1, averaged over the experts as in
+// Section 3.3, compares a prediction with what a batch did.
 // Both are one-CTA kernels: E <= 256.
 #include "common.cuh"
 
@@ -73,6 +74,7 @@ bool ok16(const void* p) { return p != nullptr && moegps_aligned16(p); }
 extern "C" MOEGPS_API int moegps_predictor_update(moegps_ctx_t* ctx, const int32_t* hist, int64_t* state,
                                                   int32_t* predicted_hist, void* stream) {
   if (!ctx || !ok16(hist) || !ok16(state) || !ok16(predicted_hist)) return MOEGPS_ERR_INVALID_ARG;
+  if (int rc = moegps_check_device(ctx)) return rc;
   predictor_update_kernel<<<1, kThreads, 0, (cudaStream_t)stream>>>(hist, ctx->shape.E,
                                                                      reinterpret_cast<long long*>(state),
                                                                      predicted_hist, ctx->d_status);
@@ -85,6 +87,7 @@ extern "C" MOEGPS_API int moegps_error_rate(moegps_ctx_t* ctx, const int32_t* pr
   if (!ctx || !ok16(predicted_hist) || !ok16(hist) || !error_rate ||
       (reinterpret_cast<uintptr_t>(error_rate) & 7u))
     return MOEGPS_ERR_INVALID_ARG;
+  if (int rc = moegps_check_device(ctx)) return rc;
   error_rate_kernel<<<1, kThreads, 0, (cudaStream_t)stream>>>(predicted_hist, hist, ctx->shape.E, error_rate);
   MOEGPS_AFTER_LAUNCH(ctx);
   return MOEGPS_OK;

@@ -26,6 +26,7 @@ __global__ void bounded_wait_kernel(long long limit_cycles, int32_t* __restrict_
 
 extern "C" MOEGPS_API int moegps_selftest_bounded_wait(moegps_ctx_t* ctx, int64_t limit_cycles, void* stream) {
   if (!ctx || limit_cycles < 1000 || limit_cycles > 4000000000ll) return MOEGPS_ERR_INVALID_ARG;
+  if (int rc = moegps_check_device(ctx)) return rc;
   bounded_wait_kernel<<<1, 32, 0, (cudaStream_t)stream>>>((long long)limit_cycles, ctx->d_status);
   MOEGPS_AFTER_LAUNCH(ctx);
   return MOEGPS_OK;

@@ -43,6 +43,16 @@ ROUTE_CASES = [
     small("fine_grained", T=64, D=256, E=200, K=8, S=200),
     small("tiny", T=65, D=64, E=5, K=5, S=5),
     small("tiny", T=40, D=64, E=33, K=1, S=40, gate_mode=1),
+    # few token tiles and a long model dimension: the launcher splits D over clusters of eight CTAs
+    # (at most 23 tiles of 128 tokens and D >= 2048), the widest split-K reduction
+    small("mixtral", T=1024, D=4096),
+    small("mixtral", T=2944, D=7168, gate_mode=1),
+    small("many_expert", T=128, D=2048),
+    small("many_expert", T=1000, D=4096, gate_mode=1),
+    small("fine_grained", T=2944, D=7168),
+    small("fine_grained", T=1024, D=2048, gate_mode=0),
+    # four-CTA clusters with E = 256 and a ragged last tile
+    small("fine_grained", T=3001, D=4096),
 ]
 
 
@@ -249,11 +259,16 @@ FFN_CASES = [
     (700, 128, 1408, 16, 4, 20, 128, 1.2),     # several row tiles per slot, F = 11 x 128
     (64, 64, 64, 32, 8, 40, 128, 1.0),         # many almost-empty slots
     (5, 2048, 256, 2, 1, 2, 128, 0.0),         # long K loop, a handful of rows
-    # long slots: many row tiles per slot, more tiles than CTAs (several rounds of the persistent loop)
+    # long slots: many row tiles per slot
     (1500, 256, 384, 2, 2, 3, 128, 0.5),
     (1500, 256, 384, 2, 2, 3, 1, 0.5),         # unaligned slots: row tiles straddle slot ends
     (3000, 128, 256, 4, 1, 4, 128, 1.5),       # one hot slot with many row tiles, cold ones with one
     (1100, 200, 328, 2, 1, 2, 128, 0.0),       # ragged K and N tails with several row tiles
+    # far more tiles than CTAs: gate+up about 1550 tiles and down about 780 (a persistent CTA walks
+    # 5-11 tiles of 16 K-blocks each, so the shared-memory ring and the two accumulators wrap many times)
+    (12288, 1024, 1024, 8, 2, 8, 128, 0.8),
+    (12288, 1024, 1024, 8, 2, 12, 1, 0.8),     # the same with unaligned slots and replicas
+    (6000, 2048, 256, 4, 2, 6, 128, 1.0),      # down GEMM with 8 column tiles per row tile, 32 K-blocks in gate+up
 ]
 
 
@@ -292,6 +307,37 @@ def test_expert_ffn(T, D, F, E, K, S, A, skew):
     ctx.expert_ffn(xpd, i32(sro), i32(se), w1.to(DEV), w3.to(DEV), w2.to(DEV), h_ws, yp2)
     ctx.check_status()
     assert np.array_equal(hz.bits(yp)[occ], hz.bits(yp2)[occ])
+
+
+@pytest.mark.parametrize("offsets", [[0, 128, 640], [0, -128, 128], [0, 256, 128]])
+def test_expert_ffn_skips_slot_extents_outside_the_buffers(offsets):
+    """slot_row_off that runs past Rcap, goes negative or decreases: the slots concerned are skipped
+    (nothing is read or written for them), BAD_INDEX is reported, nothing faults.  The buffers are
+    allocated longer than Rcap rows with a poisoned tail that must stay untouched."""
+    T, D, F, E = 256, 128, 256, 2
+    shape = binding.Shape(T, D, F, E, 1, E, 0, 128)            # Rcap = 510
+    ctx = binding.Context(shape)
+    g = torch.Generator().manual_seed(5)
+    rows = 1024
+    xp_all = torch.randn(rows, D, generator=g).to(torch.bfloat16).to(DEV)
+    w1 = (torch.randn(E, F, D, generator=g) / math.sqrt(D)).to(torch.bfloat16).to(DEV)
+    w3 = (torch.randn(E, F, D, generator=g) / math.sqrt(D)).to(torch.bfloat16).to(DEV)
+    w2 = (torch.randn(E, D, F, generator=g) / math.sqrt(F)).to(torch.bfloat16).to(DEV)
+    h_all, yp_all = poison_bf16(rows, F), poison_bf16(rows, D)
+    ctx.expert_ffn(xp_all[:shape.Rcap], i32(offsets), i32([0, 1]), w1, w3, w2, h_all[:shape.Rcap], yp_all[:shape.Rcap])
+    assert ctx.status() == binding.ERR_BAD_INDEX
+    sane = [s for s in range(E) if 0 <= offsets[s] <= offsets[s + 1] <= shape.Rcap]
+    written = torch.zeros(rows, dtype=torch.bool, device=DEV)
+    for s in sane:
+        written[offsets[s]:offsets[s + 1]] = True
+    assert torch.isnan(yp_all[~written]).all() and torch.isnan(h_all[~written]).all()
+    assert torch.isfinite(yp_all[written].float()).all()
+    if sane:                                                    # and the sane slot is still right
+        s = sane[0]
+        ref = oracle.expert_ffn(hz.bits(xp_all[:shape.Rcap]), [offsets[s], offsets[s + 1]], [s], hz.bits(w1), hz.bits(w3),
+                                hz.bits(w2))
+        hz.assert_close_rel_max(yp_all[offsets[s]:offsets[s + 1]].float().cpu().numpy(),
+                                ref[offsets[s]:offsets[s + 1]], "yp of the sane slot")
 
 
 def test_expert_ffn_zero_gate_weights_give_zero():

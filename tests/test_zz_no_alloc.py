@@ -12,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2506_07366_b200 import binding
 
 pytestmark = pytest.mark.gpu
@@ -19,11 +20,12 @@ DEV = "cuda"
 
 
 def routing(T, K, E, seed, skew):
+    """K distinct experts per token, popular ones more often (Gumbel top-K draw: no Python loop)."""
     rng = np.random.default_rng(seed)
-    p = 1.0 / np.arange(1, E + 1) ** skew
-    p /= p.sum()
-    idx = np.stack([rng.choice(E, size=K, replace=False, p=p) for _ in range(T)]).astype(np.int32)
-    return torch.from_numpy(idx).to(DEV)
+    logp = -skew * np.log(np.arange(1, E + 1))
+    keys = logp[None, :] + rng.gumbel(size=(T, E))
+    idx = np.argsort(-keys, axis=1)[:, :K].astype(np.int32)
+    return torch.from_numpy(np.ascontiguousarray(idx)).to(DEV)
 
 
 def run_both(ctx, shape, x, idx, pred):
@@ -41,7 +43,12 @@ def run_both(ctx, shape, x, idx, pred):
         pr = torch.full((shape.T, shape.K), -5, **i32)
         xp = torch.full((shape.Rcap, shape.D), 0x3C3C, dtype=torch.int16, device=DEV).view(torch.bfloat16)
         if static:
+            # the claim "allocates nothing": neither the driver's nor torch's view of device memory moves
+            torch.cuda.synchronize()
+            free0, alloc0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
             ctx.dispatch_static(x, idx, hist, rep, so, sro, rp, pr, xp)
+            torch.cuda.synchronize()
+            assert torch.cuda.mem_get_info()[0] == free0 and torch.cuda.memory_allocated() == alloc0
         else:
             ws = torch.empty(binding.workspace_bytes(shape), dtype=torch.uint8, device=DEV)
             ctx.dispatch(x, idx, hist, rep, so, sro, rp, pr, xp, ws)
@@ -64,6 +71,41 @@ def test_dispatch_static_matches_dispatch_twice_in_a_row():
         assert torch.equal(pr_a, pr_b), f"call {call}: pair_row"
         assert torch.equal(xp_a.view(torch.int16), xp_b.view(torch.int16)), f"call {call}: xp"
         assert int((rp_b >= 0).sum()) == shape.R          # and it really did the work
+        idx_h = idx.cpu().numpy()                         # the oracle agrees with both
+        hist = oracle.histogram(idx_h, shape.E)
+        rep, so, _, _ = oracle.plan(pred.cpu().numpy(), shape.S)
+        sro_ref, rp_ref, pr_ref, _ = oracle.dispatch(None, idx_h, hist, rep, so, shape.S, shape.row_align)
+        assert np.array_equal(sro_b.cpu().numpy(), sro_ref) and np.array_equal(rp_b.cpu().numpy(), rp_ref)
+        assert np.array_equal(pr_b.cpu().numpy(), pr_ref)
+
+
+@pytest.mark.parametrize("T,D,E,K,S,A", [
+    (32768, 8, 256, 8, 256, 1),     # ceil(T*K/256) * E = 262144: exactly the scratch, 1024 segments
+    (45000, 16, 16, 6, 20, 16),     # 1055 segments: the path that scans the counts on the device
+    (131073, 8, 3, 2, 7, 1),        # 1025 segments, a ragged last one
+])
+def test_dispatch_static_at_its_limit_and_on_the_scan_path(T, D, E, K, S, A):
+    """Bit-exact against moegps_dispatch AND against the oracle, twice in a row."""
+    shape = binding.Shape(T=T, D=D, F=8, E=E, K=K, S=S, gate_mode=0, row_align=A)
+    ctx = binding.Context(shape)
+    g = torch.Generator().manual_seed(T)
+    for call in range(2):
+        x = torch.randn(T, D, generator=g).to(torch.bfloat16).to(DEV)
+        idx = routing(T, K, E, 100 + call, 1.0)
+        pred = torch.bincount(idx.reshape(-1).long(), minlength=E).to(torch.int32)
+        (sro_a, rp_a, pr_a, xp_a), (sro_b, rp_b, pr_b, xp_b) = run_both(ctx, shape, x, idx, pred)
+        assert torch.equal(sro_a, sro_b) and torch.equal(rp_a, rp_b) and torch.equal(pr_a, pr_b)
+        assert torch.equal(xp_a.view(torch.int16), xp_b.view(torch.int16))
+        idx_h = idx.cpu().numpy()
+        hist = oracle.histogram(idx_h, E)
+        rep, so, _, _ = oracle.plan(hist, S)
+        sro_ref, rp_ref, pr_ref, _ = oracle.dispatch(None, idx_h, hist, rep, so, S, A)
+        assert np.array_equal(sro_b.cpu().numpy(), sro_ref)
+        assert np.array_equal(rp_b.cpu().numpy(), rp_ref)
+        assert np.array_equal(pr_b.cpu().numpy(), pr_ref)
+        occ = torch.from_numpy(rp_ref >= 0).to(DEV)
+        src = torch.from_numpy(rp_ref[rp_ref >= 0] // K).to(DEV)
+        assert torch.equal(xp_b[occ].view(torch.int16), x[src].view(torch.int16))
 
 
 def test_dispatch_static_rejects_oversized_problem():
