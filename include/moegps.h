@@ -126,6 +126,28 @@ MOEGPS_API int moegps_histogram(moegps_ctx_t* ctx, const int32_t* topk_idx, int3
 MOEGPS_API int moegps_plan(moegps_ctx_t* ctx, const int32_t* predicted_hist, int32_t n_slots,
                 int32_t* replicas, int32_t* slot_off, int32_t* slot_expert, int32_t* bound, void* stream);
 
+/* pack - Algorithm 1 of the paper as printed (Section 3.1): G devices, each with room for
+ * capacity[g] expert copies (all experts are the same size, so the algorithm's memory test is a
+ * count of free places), several experts per device, at most c_max copies of an expert (shape.c_max;
+ * 0 = no cap).  Only predicted counts are known before routing (Section 3.2.1), so the dispatch is
+ * kept as counts: share[e,g] = tokens of expert e served by device g.  Start: expert e alone on
+ * home[e] with all its tokens.  While max_g L_g - min_g L_g > 1: g_h / g_c = most / least loaded
+ * device (ties: lowest index), Delta = ceil((L_gh - L_gc)/2), e* = the expert with the most tokens on
+ * g_h (ties: lowest index) among those g_c hosts or may still receive; copy e* to g_c if needed and
+ * move min(Delta, share[e*,g_h]) of its tokens.  Ends when the loads differ by at most one token or
+ * g_c can serve no expert of g_h (the printed algorithm leaves that case open).
+ * predicted_hist: int32 [E] >= 0; home: int32 [E] in [0,G); capacity: int32 [G] (>= the experts homed
+ * there); n_devices = G in [1,64].
+ * placement: int32 [E,G] of 0/1; share: int32 [E,G]; load: int32 [G] (column sums of share);
+ * iterations: int32 [1] (moves made).  All device pointers, 16-byte aligned (iterations: 4).
+ * A home outside [0,G), a negative count or an over-full initial placement is reported as
+ * MOEGPS_ERR_BAD_INDEX and the outputs then describe the (clamped) initial placement.
+ * This call plans only: mapping its placement onto devices and the all-to-all between them are not
+ * part of this single-device library. */
+MOEGPS_API int moegps_pack(moegps_ctx_t* ctx, const int32_t* predicted_hist, const int32_t* home,
+                           const int32_t* capacity, int32_t n_devices, int32_t* placement, int32_t* share,
+                           int32_t* load, int32_t* iterations, void* stream);
+
 /* dispatch - the routing shuffle (paper, Section 2 all-to-all; Algorithm 1's dispatch d and its
  * "first tokens" rule): pairs of expert e, in flat pair order, are split into r_e contiguous
  * balanced ranges (replica rho takes stable ranks floor(rho*n_e/r_e) .. floor((rho+1)*n_e/r_e)-1)

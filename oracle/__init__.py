@@ -15,6 +15,7 @@ from .moe_oracle import (  # noqa: F401
     error_rate,
     predictor_update,
     plan,
+    pack,
     replica_starts,
     dispatch,
     expert_ffn,

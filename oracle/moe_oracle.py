@@ -24,7 +24,7 @@ import numpy as np
 __all__ = [
     "bf16_bits_to_f64", "route_logits", "route", "histogram", "p_hat", "skewness", "error_rate",
     "predictor_update",
-    "plan", "replica_starts", "dispatch", "expert_ffn", "combine", "moe_layer",
+    "plan", "pack", "replica_starts", "dispatch", "expert_ffn", "combine", "moe_layer",
 ]
 
 
@@ -202,6 +202,80 @@ def plan(pred_hist, S: int, c_max: int = 0):
     bound = max(-(-n[e] // r[e]) for e in range(E))
     return (np.array(r, dtype=np.int32), np.array(slot_off, dtype=np.int32),
             np.array(slot_expert, dtype=np.int32), int(bound))
+
+
+# --------------------------------------------------------------------------------------------
+# pack  (Algorithm 1 itself: G devices with limited memory, several experts per device)
+# --------------------------------------------------------------------------------------------
+def pack(pred_hist, home, capacity, c_max: int = 0, max_iters: int = 1 << 20):
+    """Algorithm 1 on predicted per-expert token counts, in count form.
+
+    Devices g = 0..G-1 can hold capacity[g] expert copies each (all experts have the same number of
+    parameters, so the algorithm's memory test "params(e) <= M_g" is a count of free places).  The
+    initial placement puts expert e on device home[e] alone, and all its n_e tokens are dispatched
+    there (the algorithm's first step: every token goes to the lowest device that hosts its expert).
+    Only counts are known before routing (Section 3.2.1), so the dispatch d is kept as
+    share[e][g] = number of expert e's tokens served by device g, and "the first Delta tokens" are
+    any Delta of them.
+
+    Loop, exactly as printed, while max_g L_g - min_g L_g > 1:
+      g_h = argmax L, g_c = argmin L (ties: lowest device);  Delta = ceil((L_gh - L_gc) / 2);
+      e* = the expert with the most tokens on g_h (ties: lowest expert) AMONG those that g_c already
+           hosts or may receive: copies(e) < c_max (c_max = 0: no cap) and g_c has a free place;
+      copy e* to g_c if it is not there;  move min(Delta, share[e*][g_h]) tokens of e* from g_h to g_c.
+    The restriction of e* to experts that g_c can serve is the reading taken where the printed
+    algorithm is incomplete: as printed, a refused copy would still send tokens to a device without
+    the expert.  When no expert of g_h can be served by g_c the loop ends (no legal move for the
+    hottest/coldest pair).  Every pass moves between 1 and Delta < L_gh - L_gc tokens, so
+    sum_g L_g^2 falls strictly and the loop terminates.
+
+    Returns (placement int32 [E, G] of 0/1, share int64 [E, G], load int64 [G], iterations).
+    """
+    n = [int(v) for v in np.asarray(pred_hist).reshape(-1)]
+    hm = [int(v) for v in np.asarray(home).reshape(-1)]
+    cap = [int(v) for v in np.asarray(capacity).reshape(-1)]
+    E, G = len(n), len(cap)
+    if len(hm) != E or any(v < 0 for v in n) or any(not (0 <= g < G) for g in hm):
+        raise ValueError("need counts >= 0 and a home device in [0, G) per expert")
+    placed = [[0] * G for _ in range(E)]
+    share = [[0] * G for _ in range(E)]
+    used = [0] * G
+    copies = [1] * E
+    for e in range(E):
+        placed[e][hm[e]] = 1
+        share[e][hm[e]] = n[e]
+        used[hm[e]] += 1
+    if any(used[g] > cap[g] for g in range(G)):
+        raise ValueError("the initial placement exceeds a device's capacity")
+    load = [sum(share[e][g] for e in range(E)) for g in range(G)]
+    iters = 0
+    while iters < max_iters:
+        g_h = max(range(G), key=lambda g: (load[g], -g))
+        g_c = min(range(G), key=lambda g: (load[g], g))
+        if load[g_h] - load[g_c] <= 1:
+            break
+        delta = -(-(load[g_h] - load[g_c]) // 2)
+        best = -1
+        for e in range(E):
+            if share[e][g_h] <= 0:
+                continue
+            servable = placed[e][g_c] or ((c_max <= 0 or copies[e] < c_max) and used[g_c] < cap[g_c])
+            if servable and (best < 0 or share[e][g_h] > share[best][g_h]):
+                best = e
+        if best < 0:
+            break
+        if not placed[best][g_c]:
+            placed[best][g_c] = 1
+            copies[best] += 1
+            used[g_c] += 1
+        m = min(delta, share[best][g_h])
+        share[best][g_h] -= m
+        share[best][g_c] += m
+        load[g_h] -= m
+        load[g_c] += m
+        iters += 1
+    return (np.array(placed, dtype=np.int32), np.array(share, dtype=np.int64),
+            np.array(load, dtype=np.int64), iters)
 
 
 # --------------------------------------------------------------------------------------------

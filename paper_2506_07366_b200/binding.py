@@ -53,7 +53,7 @@ ERR_STATIC_SCRATCH_EXCEEDED = -9
 
 EXPORTS = (
     "moegps_create", "moegps_destroy", "moegps_rcap", "moegps_workspace_bytes", "moegps_route",
-    "moegps_route_histogram", "moegps_route_logits", "moegps_histogram", "moegps_plan", "moegps_dispatch", "moegps_dispatch_static",
+    "moegps_route_histogram", "moegps_route_logits", "moegps_histogram", "moegps_plan", "moegps_pack", "moegps_dispatch", "moegps_dispatch_static",
     "moegps_expert_ffn", "moegps_expert_ffn_gate_up", "moegps_expert_ffn_down", "moegps_combine",
     "moegps_status", "moegps_launch_count", "moegps_last_cuda_error", "moegps_error_string",
     "moegps_selftest_bounded_wait", "moegps_predictor_update", "moegps_error_rate",
@@ -98,6 +98,7 @@ def _lib():
         "moegps_route_logits": (ctypes.c_int, [vp] * 6),
         "moegps_histogram": (ctypes.c_int, [vp] * 4),
         "moegps_plan": (ctypes.c_int, [vp, vp, i32, vp, vp, vp, vp, vp]),
+        "moegps_pack": (ctypes.c_int, [vp, vp, vp, vp, i32, vp, vp, vp, vp, vp]),
         "moegps_dispatch": (ctypes.c_int, [vp] * 12),
         "moegps_dispatch_static": (ctypes.c_int, [vp] * 11),
         "moegps_expert_ffn": (ctypes.c_int, [vp] * 10),
@@ -217,6 +218,15 @@ class Context:
             _ptr(slot_off, torch.int32, (s.E + 1,), "slot_off"),
             _ptr(slot_expert, torch.int32, (s.S,), "slot_expert"),
             _ptr(bound, torch.int32, (1,), "bound"), _stream(stream)), "moegps_plan")
+
+    def pack(self, predicted_hist, home, capacity, n_devices, placement, share, load, iterations, stream=None):
+        s, g = self.shape, int(n_devices)
+        self._check(_lib().moegps_pack(
+            self._h, _ptr(predicted_hist, torch.int32, (s.E,), "predicted_hist"),
+            _ptr(home, torch.int32, (s.E,), "home"), _ptr(capacity, torch.int32, (g,), "capacity"), g,
+            _ptr(placement, torch.int32, (s.E, g), "placement"), _ptr(share, torch.int32, (s.E, g), "share"),
+            _ptr(load, torch.int32, (g,), "load"), _ptr(iterations, torch.int32, (1,), "iterations"),
+            _stream(stream)), "moegps_pack")
 
     def dispatch(self, x, topk_idx, hist, replicas, slot_off, slot_row_off, row_pair, pair_row, xp,
                  workspace, stream=None):

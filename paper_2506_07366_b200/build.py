@@ -10,7 +10,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libmoegps.so")
-SOURCES = ["api.cu", "route.cu", "histogram.cu", "plan.cu", "dispatch.cu", "expert_ffn.cu", "combine.cu",
+SOURCES = ["api.cu", "route.cu", "histogram.cu", "plan.cu", "pack.cu", "dispatch.cu", "expert_ffn.cu", "combine.cu",
            "predictor.cu", "selftest.cu"]
 HEADERS = ["common.cuh", "sm100.cuh", "route_epilogue.cuh"]
 

@@ -46,10 +46,11 @@ int moegps_create(moegps_ctx_t** out, const moegps_shape_t* shape, int device) {
   ctx->last_cuda_error = 0;
   ctx->tm1_valid = false;
   ctx->tm2_valid = false;
-  ctx->ffn_attr_done = false;
+  for (bool& b : ctx->ffn_attr_done) b = false;
   ctx->rt_valid = false;
   ctx->route_attr_done = false;
   ctx->dispatch_attr_done = false;
+  ctx->pack_attr_done = false;
   ctx->d_status = nullptr;
   int prev = 0;
   cudaGetDevice(&prev);

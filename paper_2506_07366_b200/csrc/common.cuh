@@ -23,13 +23,14 @@ struct moegps_ctx {
   const void* tm_key2[2];   // h_ws, w_down
   CUtensorMap tm_h, tm_w2;
   bool tm2_valid;
-  bool ffn_attr_done;    // dynamic shared-memory limit of the GEMM kernels raised on this device
+  bool ffn_attr_done[2]; // dynamic shared-memory limit raised: gate+up and down instantiations of the GEMM kernel
   // cached TMA descriptors of the router
   const void* rt_key[2];
   CUtensorMap tm_rx, tm_rw;
   bool rt_valid;
   bool route_attr_done;
   bool dispatch_attr_done;
+  bool pack_attr_done;
 };
 
 #define MOEGPS_CUDA_TRY(ctx, expr)                                   \

@@ -9,6 +9,12 @@
 // i) are handed around with mbarriers; every wait is bounded and raises an abort flag on expiry.
 // Tiles are enumerated on the device from slot_row_off (no host round trip): slot-major, then
 // column tile, then row tile, so that CTAs working at the same time share weight tiles in L2.
+//
+// The launch shape is a template parameter (ring depth, accumulators, epilogue warps, CTAs per SM).
+// One shape is in use: 1 CTA per SM, 4-stage ring, two accumulators, 8 epilogue warps.  A shape with
+// two smaller CTAs per SM (2-stage rings, one accumulator and 4 epilogue warps each), meant to let a
+// weight-streaming tile of a short slot overlap a tensor-bound tile of a long slot on one SM, was
+// measured 3-9 % slower on every workload (halving each ring costs more than the overlap returns).
 #include "common.cuh"
 #include "sm100.cuh"
 
@@ -26,23 +32,36 @@ constexpr int BNACC = 256;         // accumulator columns per tile
 // rows far more efficiently, which outweighs the deeper ring.
 constexpr int BK = MOEGPS_FFN_BK;
 constexpr int kRowBytes = BK * 2;
-constexpr int kStages = 256 / BK;  // 192 KiB of ring either way
 constexpr int kABytes = BM * BK * 2;
 constexpr int kBHalfBytes = 128 * BK * 2;
 constexpr int kStageBytes = kABytes + 2 * kBHalfBytes;       // 48 KiB
-constexpr int kThreads = 320;      // producer warp, MMA warp, 8 epilogue warps (two per TMEM lane quarter)
 constexpr int kMaxS = 1024;
-constexpr int kTmemCols = 512;
 
+template <int kStages_, int kAccs_, int kEpiWarps_, int kCtasPerSm_>
+struct GemmCfg {
+  static constexpr int kStages = kStages_;        // ring depth (48 KiB per stage)
+  static constexpr int kAccs = kAccs_;            // 256-column TMEM accumulators
+  static constexpr int kEpiWarps = kEpiWarps_;    // 4: one per TMEM lane quarter; 8: two per quarter, half the columns each
+  static constexpr int kCtasPerSm = kCtasPerSm_;
+  static constexpr int kThreads = 64 + 32 * kEpiWarps_;   // producer warp, MMA warp, epilogue warps
+  static constexpr int kTmemCols = 256 * kAccs_;
+};
+using WideCfg = GemmCfg<256 / BK, 2, 8, 1>;       // 192 KiB of ring
+
+// Per-CTA copy of what decoding a tile needs.  tile_base[s] = first tile index of slot s.
 struct __align__(16) Tables {
-  int32_t tile_base[kMaxS + 1];    // first tile index of each slot
-  int32_t row_off[kMaxS + 1];
-  int32_t expert[kMaxS];
+  int32_t tile_base[kMaxS + 1];
 };
 
-constexpr int kEpilogueWarps = 8;
-constexpr size_t kSmemBytes = 1024 /* alignment slack */ + (size_t)kStages * kStageBytes + sizeof(Tables) + 256 +
-                              kEpilogueWarps * 32 * 80 /* epilogue staging */;
+constexpr int kStageRowBytes = 80;                 // epilogue staging: 64 payload bytes per row, conflict-free pitch
+constexpr int kStagingBytesPerWarp = 32 * kStageRowBytes;
+
+template <class Cfg>
+constexpr size_t smem_bytes_of() {
+  return 1024 /* alignment slack */ + (size_t)Cfg::kStages * kStageBytes + sizeof(Tables) + 256 +
+         (size_t)Cfg::kEpiWarps * kStagingBytesPerWarp;
+}
+static_assert(smem_bytes_of<WideCfg>() <= 227 * 1024, "one CTA per SM");
 
 struct TileCoord {
   int m0;        // first row of the tile in the permuted buffer
@@ -51,7 +70,8 @@ struct TileCoord {
   int expert;
 };
 
-__device__ __forceinline__ TileCoord decode_tile_rows(const Tables& tb, int S, int tile, int n_tiles, int tile_rows) {
+__device__ __forceinline__ TileCoord decode_tile(const Tables& tb, const int32_t* __restrict__ slot_row_off,
+                                               const int32_t* __restrict__ slot_expert, int S, int tile, int n_tiles) {
   int lo = 0, hi = S;                 // find s with tile_base[s] <= tile < tile_base[s+1]
   while (hi - lo > 1) {
     const int mid = (lo + hi) >> 1;
@@ -62,14 +82,12 @@ __device__ __forceinline__ TileCoord decode_tile_rows(const Tables& tb, int S, i
   const int mt = (tb.tile_base[s + 1] - tb.tile_base[s]) / n_tiles;   // row tiles of this slot
   TileCoord c;
   c.n_tile = local / mt;
-  c.m0 = tb.row_off[s] + (local % mt) * tile_rows;
-  c.row_end = tb.row_off[s + 1];
-  c.expert = tb.expert[s];
+  // (the slot tables are a few KiB that every CTA reads: they stay in L1/L2; only slots that passed
+  // the checks of the table build own tiles, so these values are in range)
+  c.m0 = __ldg(slot_row_off + s) + (local % mt) * BM;
+  c.row_end = __ldg(slot_row_off + s + 1);
+  c.expert = __ldg(slot_expert + s);
   return c;
-}
-
-__device__ __forceinline__ TileCoord decode_tile(const Tables& tb, int S, int tile, int n_tiles) {
-  return decode_tile_rows(tb, S, tile, n_tiles, BM);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -88,21 +106,17 @@ __device__ __forceinline__ float silu_fast(float g) {
 // Epilogue of one tile for one warp: 32 accumulator rows (one per lane) x half of the tile's output
 // columns, TMEM -> registers -> bf16 -> shared-memory staging -> global.
 // kSwiGLU: columns [0,128) are the gate and [128,256) the up projection; 128 outputs silu(g)*u.
-// `half` (0 or 1) selects which half of the output columns this warp drains (two warps share each
-// quarter of the TMEM lanes).  A lane owns one row, so storing straight from registers would
+// [c_begin, c_end) are the output columns this warp drains (with eight epilogue warps two share each
+// quarter of the TMEM lanes and take half the columns each).  A lane owns one row, so storing straight from registers would
 // scatter 16-byte pieces over 32 rows per instruction - measured to cost the main loop 5-14 % of its
 // L2/HBM throughput.  Instead each 32-column chunk (64 bytes per row) goes through a per-warp
 // staging buffer (rows 80 bytes apart: conflict-free) and is written out with four lanes per row,
 // i.e. whole 64-byte segments.  `row0` is the first of the warp's 32 rows, `row_end` the slot's end.
-constexpr int kStageRowBytes = 80;
-constexpr int kStagingBytesPerWarp = 32 * kStageRowBytes;
-
 template <bool kSwiGLU>
 __device__ __forceinline__ void drain_tile(uint32_t taddr, uint8_t* staging, int lane, __nv_bfloat16* out,
-                                           int row0, int row_end, int col0, int n_dim, int half) {
-  constexpr int kCols = kSwiGLU ? 128 : 256;          // output columns of a tile
+                                           int row0, int row_end, int col0, int n_dim, int c_begin, int c_end) {
 #pragma unroll 1
-  for (int c0 = (kCols / 2) * half; c0 < (kCols / 2) * (half + 1); c0 += 32) {
+  for (int c0 = c_begin; c0 < c_end; c0 += 32) {
     uint32_t o[16];
     if constexpr (kSwiGLU) {
       uint32_t g[32], u[32];
@@ -140,12 +154,13 @@ __device__ __forceinline__ void drain_tile(uint32_t taddr, uint8_t* staging, int
 
 // kSwiGLU = true : out[row, n_tile*128 + c] = silu(acc[c]) * acc[128 + c],  c < 128
 // kSwiGLU = false: out[row, n_tile*256 + c] = acc[c],                        c < 256
-template <bool kSwiGLU>
-__global__ void __launch_bounds__(kThreads, 1)
+template <bool kSwiGLU, class Cfg>
+__global__ void __launch_bounds__(Cfg::kThreads, Cfg::kCtasPerSm)
 grouped_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
                     const __grid_constant__ CUtensorMap tm_b1, const int32_t* __restrict__ slot_row_off,
                     const int32_t* __restrict__ slot_expert, int S, int E, int n_dim, int k_dim, int rcap,
                     __nv_bfloat16* __restrict__ out, int32_t* __restrict__ status) {
+  constexpr int kStages = Cfg::kStages, kAccs = Cfg::kAccs, kThreads = Cfg::kThreads;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* stage_mem = smem;                                          // kStages x (A | B0 | B1), 1024-aligned
@@ -153,11 +168,11 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kStages * kStageBytes + sizeof(Tables));
   uint64_t* full = bars;                  // [kStages]  TMA -> MMA
   uint64_t* empty = bars + kStages;       // [kStages]  MMA -> TMA
-  uint64_t* acc_full = bars + 2 * kStages;       // [2]  MMA -> epilogue
-  uint64_t* acc_empty = bars + 2 * kStages + 2;  // [2]  epilogue -> MMA
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
+  uint64_t* acc_full = bars + 2 * kStages;           // [kAccs]  MMA -> epilogue
+  uint64_t* acc_empty = bars + 2 * kStages + kAccs;  // [kAccs]  epilogue -> MMA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 2 * kAccs);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  int* total_tiles_p = const_cast<int*>(reinterpret_cast<volatile int*>(tmem_slot + 2));
+  int* warp_tiles = const_cast<int*>(reinterpret_cast<volatile int*>(tmem_slot + 2));   // [32] scan scratch
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cols_per_tile = kSwiGLU ? 128 : 256;
@@ -165,11 +180,9 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
   const int num_kb = (k_dim + BK - 1) / BK;
 
   // ---------------------------------------------------------------- set-up
-  for (int s = threadIdx.x; s <= S; s += kThreads) tb.row_off[s] = slot_row_off[s];
-  for (int s = threadIdx.x; s < S; s += kThreads) tb.expert[s] = slot_expert[s];
   if (threadIdx.x == 0) {
     for (int i = 0; i < kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 8); }
+    for (int i = 0; i < kAccs; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], Cfg::kEpiWarps); }
     *abort_flag = 0;
     fence_mbar_init();
     prefetch_tensormap(&tm_a);
@@ -177,33 +190,57 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     prefetch_tensormap(&tm_b1);
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, kTmemCols);
+    tmem_alloc(tmem_slot, Cfg::kTmemCols);
     tmem_relinquish();
   }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    int acc = 0;
-    for (int s = 0; s < S; ++s) {
-      tb.tile_base[s] = acc;
-      // a slot whose extent is not inside [0, rcap] (offsets negative, decreasing or past the
-      // buffers) gets no tiles: nothing is read or written for it, and the caller is told
-      const int lo = tb.row_off[s], hi = tb.row_off[s + 1];
-      const int e = tb.expert[s];
+  // tiles per slot.  A slot whose extent is not inside [0, rcap] (offsets negative, decreasing or
+  // past the buffers) gets no tiles: nothing is read or written for it, and the caller is told.
+  for (int s = threadIdx.x; s <= kMaxS; s += kThreads) {
+    int cnt = 0;
+    if (s < S) {
+      const int lo = slot_row_off[s], hi = slot_row_off[s + 1];
+      const int e = slot_expert[s];
       if (lo < 0 || hi < lo || hi > rcap) {
-        moegps_report(status, MOEGPS_ERR_BAD_INDEX, s);
-        continue;
+        if (blockIdx.x == 0) moegps_report(status, MOEGPS_ERR_BAD_INDEX, s);
+      } else if (hi > lo && e >= 0 && e < E) {
+        cnt = ((hi - lo + BM - 1) / BM) * n_tiles;
+      } else if (hi > lo && e >= E) {
+        if (blockIdx.x == 0) moegps_report(status, MOEGPS_ERR_BAD_INDEX, s);
       }
-      if (hi > lo && e >= 0 && e < E) acc += ((hi - lo + BM - 1) / BM) * n_tiles;
-      else if (hi > lo && e >= E) moegps_report(status, MOEGPS_ERR_BAD_INDEX, s);
     }
-    tb.tile_base[S] = acc;
-    *total_tiles_p = acc;
+    tb.tile_base[s] = cnt;
   }
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
+  // exclusive prefix sum of the counts (warp 0: lane l owns entries 33 l .. 33 l + 32; 32 * 33 > kMaxS)
+  if (warp == 0) {
+    constexpr int kPer = (kMaxS + 1 + 31) / 32;
+    int v[kPer], sum = 0;
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) {
+      const int s = lane * kPer + i;
+      v[i] = s <= kMaxS ? tb.tile_base[s] : 0;
+      sum += v[i];
+    }
+    int incl = sum;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int o = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += o;
+    }
+    int run = incl - sum;
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) {
+      const int s = lane * kPer + i;
+      if (s <= kMaxS) tb.tile_base[s] = run;
+      run += v[i];
+    }
+    if (lane == 31) warp_tiles[0] = incl;
+  }
+  __syncthreads();
   const uint32_t tmem_base = *tmem_slot;
-  const int total_tiles = *total_tiles_p;
+  const int total_tiles = warp_tiles[0];
 
   // ---------------------------------------------------------------- roles
   if (warp == 0) {
@@ -212,7 +249,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
       uint32_t phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-        const TileCoord tc = decode_tile(tb, S, tile, n_tiles);
+        const TileCoord tc = decode_tile(tb, slot_row_off, slot_expert, S, tile, n_tiles);
         const int nb0 = tc.n_tile * cols_per_tile;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -256,7 +293,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         }
         if (!ok) break;
         mma_commit(&acc_full[acc]);              // accumulator complete
-        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        if (++acc == kAccs) { acc = 0; acc_phase ^= 1u; }
       }
       if (!ok) {
         for (int i = 0; i < 1000; ++i) __nanosleep(1000);
@@ -264,22 +301,25 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     }
   } else {
     const int quarter = warp & 3;                 // TMEM lanes this warp may read
-    const int half = (warp - 2) >> 2;             // which half of the output columns it drains
+    constexpr int kOutCols = kSwiGLU ? 128 : 256; // output columns of a tile
+    constexpr int kShare = kOutCols / (Cfg::kEpiWarps / 4);          // columns per warp of a lane quarter
+    const int c_begin = ((warp - 2) >> 2) * kShare;
     uint8_t* staging = smem + (size_t)kStages * kStageBytes + sizeof(Tables) + 256 + (warp - 2) * kStagingBytesPerWarp;
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-      const TileCoord tc = decode_tile(tb, S, tile, n_tiles);
+      const TileCoord tc = decode_tile(tb, slot_row_off, slot_expert, S, tile, n_tiles);
       if (!mbar_wait(&acc_full[acc], acc_phase, abort_flag, 256)) { ok = false; break; }
       tc_fence_after_sync();
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * BNACC;
       const int col0 = tc.n_tile * cols_per_tile;
-      drain_tile<kSwiGLU>(taddr, staging, lane, out, tc.m0 + quarter * 32, tc.row_end, col0, n_dim, half);
+      drain_tile<kSwiGLU>(taddr, staging, lane, out, tc.m0 + quarter * 32, tc.row_end, col0, n_dim, c_begin,
+                          c_begin + kShare);
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(&acc_empty[acc]);
-      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      if (++acc == kAccs) { acc = 0; acc_phase ^= 1u; }
     }
   }
 
@@ -290,7 +330,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
   if (threadIdx.x == 0 && *abort_flag) moegps_report(status, MOEGPS_ERR_TIMEOUT, (int)blockIdx.x);
   if (warp == 1) {
     tc_fence_after_sync();
-    tmem_dealloc(tmem_base, kTmemCols);
+    tmem_dealloc(tmem_base, Cfg::kTmemCols);
   }
 }
 
@@ -351,19 +391,27 @@ bool moegps_make_tmap_3d(CUtensorMap* tm, const void* base, uint64_t batch, uint
 
 namespace {
 
-int raise_smem_limit(moegps_ctx* ctx) {
-  if (ctx->ffn_attr_done) return MOEGPS_OK;
-  MOEGPS_CUDA_TRY(ctx, cudaFuncSetAttribute(grouped_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            (int)kSmemBytes));
-  MOEGPS_CUDA_TRY(ctx, cudaFuncSetAttribute(grouped_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            (int)kSmemBytes));
-  ctx->ffn_attr_done = true;
-  return MOEGPS_OK;
-}
-
 int tmap_failed(moegps_ctx* ctx) {
   ctx->last_cuda_error = (int)cudaErrorInvalidValue;
   return MOEGPS_ERR_CUDA;
+}
+
+template <bool kSwiGLU, class Cfg>
+int launch_gemm(moegps_ctx* ctx, bool* attr_done, const CUtensorMap& ta, const CUtensorMap& tb0, const CUtensorMap& tb1,
+                const int32_t* slot_row_off, const int32_t* slot_expert, int n_dim, int k_dim, void* out,
+                cudaStream_t st) {
+  const moegps_shape_t& s = ctx->shape;
+  constexpr size_t smem = smem_bytes_of<Cfg>();
+  if (!*attr_done) {
+    MOEGPS_CUDA_TRY(ctx, cudaFuncSetAttribute(grouped_gemm_kernel<kSwiGLU, Cfg>,
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    *attr_done = true;
+  }
+  grouped_gemm_kernel<kSwiGLU, Cfg><<<ctx->sm_count * Cfg::kCtasPerSm, Cfg::kThreads, smem, st>>>(
+      ta, tb0, tb1, slot_row_off, slot_expert, s.S, s.E, n_dim, k_dim, (int)moegps_rcap_of(s),
+      static_cast<__nv_bfloat16*>(out), ctx->d_status);
+  MOEGPS_AFTER_LAUNCH(ctx);
+  return MOEGPS_OK;
 }
 
 }  // namespace
@@ -382,13 +430,8 @@ int moegps_launch_ffn_gate_up(moegps_ctx* ctx, const void* xp, const int32_t* sl
     ctx->tm_key1[0] = xp; ctx->tm_key1[1] = w_gate; ctx->tm_key1[2] = w_up;
     ctx->tm1_valid = true;
   }
-  int rc = raise_smem_limit(ctx);
-  if (rc != MOEGPS_OK) return rc;
-  grouped_gemm_kernel<true><<<ctx->sm_count, kThreads, kSmemBytes, st>>>(
-      ctx->tm_xp, ctx->tm_w1, ctx->tm_w3, slot_row_off, slot_expert, s.S, s.E, s.F, s.D, (int)rcap,
-      static_cast<__nv_bfloat16*>(h_ws), ctx->d_status);
-  MOEGPS_AFTER_LAUNCH(ctx);
-  return MOEGPS_OK;
+  return launch_gemm<true, WideCfg>(ctx, &ctx->ffn_attr_done[0], ctx->tm_xp, ctx->tm_w1, ctx->tm_w3, slot_row_off,
+                                    slot_expert, s.F, s.D, h_ws, st);
 }
 
 int moegps_launch_ffn_down(moegps_ctx* ctx, const void* h_ws, const int32_t* slot_row_off,
@@ -403,11 +446,6 @@ int moegps_launch_ffn_down(moegps_ctx* ctx, const void* h_ws, const int32_t* slo
     ctx->tm_key2[0] = h_ws; ctx->tm_key2[1] = w_down;
     ctx->tm2_valid = true;
   }
-  int rc = raise_smem_limit(ctx);
-  if (rc != MOEGPS_OK) return rc;
-  grouped_gemm_kernel<false><<<ctx->sm_count, kThreads, kSmemBytes, st>>>(
-      ctx->tm_h, ctx->tm_w2, ctx->tm_w2, slot_row_off, slot_expert, s.S, s.E, s.D, s.F, (int)rcap,
-      static_cast<__nv_bfloat16*>(yp), ctx->d_status);
-  MOEGPS_AFTER_LAUNCH(ctx);
-  return MOEGPS_OK;
+  return launch_gemm<false, WideCfg>(ctx, &ctx->ffn_attr_done[1], ctx->tm_h, ctx->tm_w2, ctx->tm_w2, slot_row_off,
+                                     slot_expert, s.D, s.F, yp, st);
 }

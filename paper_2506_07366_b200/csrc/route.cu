@@ -1,19 +1,30 @@
-// route: router GEMM fused with bias, warp-shuffle top-K and the gate weights (paper, Section 2).
+// route: router GEMM fused with bias, top-K selection and the gate weights (paper, Section 2).
 //
 // logits[128 tokens, E] = X_tile * Wr^T on the 5th-generation tensor cores: the token tile is the
 // MMA's M (128 rows), the experts its N (E rounded up to 16, at most 256), accumulators in TMEM.
 // The kernel is bound by reading X once from HBM, so the grid must cover the chip even when
 // T/128 is small: the model dimension is split over the KS CTAs of a thread-block cluster
 // (grid = token tiles x KS).  Each CTA streams its slice of X and Wr through a TMA -> shared-memory
-// ring into tcgen05.mma, parks its fp32 partial logits in its own shared memory, and after a
-// cluster barrier CTA r reduces rows [r*128/KS, (r+1)*128/KS) over all KS partials through
-// distributed shared memory in a fixed order (deterministic), adds the bias and lets eight lanes per
-// token select the top K by shuffles (route_epilogue.cuh).  When the caller asks for it, the
-// per-expert token counts (Eq. 1's n_e) are accumulated on the way: every selection bumps a
-// shared-memory counter of its CTA, and each CTA adds its non-zero counters to the global
-// histogram once (integer atomics: deterministic).
+// ring into tcgen05.mma.  The producer starts streaming as soon as the barriers exist; what the
+// epilogue needs besides (bias, counters) is fetched while the stream runs.
+//
+// Split-K reduction by PUSH: CTA r of the cluster owns rows [r*128/KS, (r+1)*128/KS) of the tile.
+// The four drain warps read the CTA's fp32 partial logits from TMEM (one thread per token row) and
+// store every row straight into its owner's shared memory (st.shared::cluster; remote stores need no
+// round trip), at [source slice][row][expert].  One cluster barrier later each owner sums the KS
+// partials of its rows from its OWN shared memory in slice order (fixed: deterministic), adds the
+// bias and selects.  The partial buffers share the ring's memory, so a first cluster barrier (arrive
+// after the CTA's last MMA has completed, wait just before the first push) guarantees that no peer
+// still feeds its tensor core from the memory being overwritten; after the second barrier nobody
+// touches a peer's shared memory any more, so CTAs leave independently.
+//
+// Selection: L lanes per token select by shuffles (route_epilogue.cuh), L chosen so that the rows the
+// CTA owns occupy all sixteen warps in one pass.  When the caller asks for it, the per-expert token
+// counts (Eq. 1's n_e) are accumulated on the way: every selection bumps a shared-memory counter of
+// its CTA, and each CTA adds its non-zero counters to the global histogram once (integer atomics:
+// deterministic).
 // Warp roles in the main loop: warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
-// warps 2..5 = TMEM -> shared-memory drain.  Every mbarrier wait is bounded.
+// warps 2..5 = drain.  Every mbarrier wait is bounded.
 #include "common.cuh"
 #include "route_epilogue.cuh"
 #include "sm100.cuh"
@@ -27,7 +38,7 @@ using namespace sm100;
 
 constexpr int BM = 128;
 constexpr int BK = 64;
-constexpr int kThreads = 384;   // 12 warps: 2 feed the tensor core, 4 drain TMEM, all 12 reduce and select
+constexpr int kThreads = 512;   // 16 warps: 2 feed the tensor core, 4 drain TMEM, all 16 reduce and select
 constexpr int kABytes = BM * BK * 2;      // 16 KiB of X per stage
 
 struct RouteParams {
@@ -39,83 +50,62 @@ struct RouteParams {
   int tmem_cols;
   int ring_bytes;   // stages * (kABytes + e_pad * 128)
   int part_stride;  // floats per row of the partial-logit buffer (e_pad + 4)
+  int lanes;        // lanes per token in the selection (4, 8, 16 or 32; >= K and >= E/32)
 };
 
-// volatile keeps these loads behind the cluster barrier (also a volatile asm) and in program order.
-__device__ __forceinline__ float4 ld_cluster_f32x4(uint32_t addr) {
-  float4 v;
-  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
-               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-               : "r"(addr));
-  return v;
+__device__ __forceinline__ void st_cluster_f32x4(uint32_t addr, float a, float b, float c, float d) {
+  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d)
+               : "memory");
+}
+__device__ __forceinline__ void cluster_arrive_release() {
+  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait_acquire() {
+  asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
 }
 
-// Split-K reduction: CTA `rank` of the cluster owns rows [rank*128/KS, (rank+1)*128/KS) of the tile.
-// All threads sum the KS partial logits of those rows in slice order (fixed: deterministic), 16
-// bytes per load - consecutive threads read consecutive chunks of a peer's shared memory - and store
-// the sums over the CTA's own partials of those rows, which no peer reads.
-template <int KS>
-__device__ __forceinline__ void reduce_partials(const RouteParams& p, float* partial, uint32_t rank) {
-  constexpr int rows_per = BM / KS;
-  const int chunks = p.e_pad / 4;
-  uint32_t peer[KS];
-#pragma unroll
-  for (int k = 0; k < KS; ++k) peer[k] = map_to_cta(smem_u32(partial), (uint32_t)k);
-  // two chunks per thread and iteration: 2*KS independent 16-byte loads in flight hide the latency of
-  // a peer's shared memory
-  const int total = rows_per * chunks;
-  for (int idx = threadIdx.x; idx < total; idx += 2 * kThreads) {
-    const int idx1 = idx + kThreads;
-    const bool two = idx1 < total;
-    const int word0 = ((int)rank * rows_per + idx / chunks) * p.part_stride + 4 * (idx % chunks);
-    const int word1 = two ? ((int)rank * rows_per + idx1 / chunks) * p.part_stride + 4 * (idx1 % chunks) : word0;
-    float4 a[KS], b[KS];
-#pragma unroll
-    for (int k = 0; k < KS; ++k) a[k] = ld_cluster_f32x4(peer[k] + (uint32_t)word0 * 4u);
-#pragma unroll
-    for (int k = 0; k < KS; ++k) b[k] = ld_cluster_f32x4(peer[k] + (uint32_t)word1 * 4u);
-    float4 sa = a[0], sb = b[0];
-#pragma unroll
-    for (int k = 1; k < KS; ++k) {
-      sa.x += a[k].x; sa.y += a[k].y; sa.z += a[k].z; sa.w += a[k].w;
-      sb.x += b[k].x; sb.y += b[k].y; sb.z += b[k].z; sb.w += b[k].w;
-    }
-    *reinterpret_cast<float4*>(partial + word0) = sa;
-    if (two) *reinterpret_cast<float4*>(partial + word1) = sb;
-  }
-}
-
-// Eight lanes per token, four tokens per warp at a time: read the row's logits (already summed
-// over the K slices) from shared memory, add the bias, turn the row into order keys (sub-lane l
-// holds experts l, l+8, ...) and select.  Every lane of a warp takes part in every shuffle, so rows
-// past T (ragged last tile; their logits are zero-filled, finite) are computed like the others and
-// only their stores are skipped.
-template <int NPL>
-__device__ __forceinline__ void select_rows(const RouteParams& p, const float* partial, int row_begin, int rows,
-                                            int m0, const float* s_bias, int32_t* __restrict__ topk_idx,
-                                            float* __restrict__ topk_w, float* __restrict__ logits_out,
+// L lanes per token, 32/L tokens per warp at a time: read the row's logits (already summed over the
+// K slices, bias added) from shared memory, turn them into order keys (sub-lane l holds experts
+// l, l+L, ...) and select.  Every lane of a warp takes part in every shuffle, so rows past T (ragged
+// last tile; their logits are zero-filled, finite) are computed like the others and only their
+// stores are skipped.
+template <int L, int NPL>
+__device__ __forceinline__ void select_rows(const RouteParams& p, const float* rows_smem, int rows, int t0,
+                                            int32_t* __restrict__ topk_idx, float* __restrict__ topk_w,
                                             int32_t* cta_hist) {
+  constexpr int kRowsPerWarp = 32 / L;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int sl = lane & 7, grp = lane >> 3;
-  for (int r0 = warp * 4; r0 < rows; r0 += (kThreads / 32) * 4) {     // rows is a multiple of 4
-    const int row = row_begin + r0 + grp;
-    const int t = m0 + row;
+  const int sl = lane & (L - 1), grp = lane / L;
+  for (int r0 = warp * kRowsPerWarp; r0 < rows; r0 += (kThreads / 32) * kRowsPerWarp) {   // rows % 8 == 0
+    const int row = r0 + grp;
+    const int t = t0 + row;
     const bool live = t < p.T;
-    const float* prow = partial + (size_t)row * p.part_stride;
+    const float* prow = rows_smem + (size_t)row * p.part_stride;
     uint32_t key[NPL];
 #pragma unroll
     for (int i = 0; i < NPL; ++i) {
-      const int e = sl + 8 * i;
-      const float v = prow[e < p.E ? e : 0] + s_bias[e < p.E ? e : 0];
-      key[i] = e < p.E ? route_order_key(v) : 0u;
-      if (logits_out && live && e < p.E) logits_out[(int64_t)t * p.E + e] = v;
+      const int e = sl + L * i;
+      key[i] = e < p.E ? route_order_key(prow[e]) : 0u;
     }
-    if (topk_idx) {
-      const int sel = group8_topk_gate<NPL>(key, p.K, p.gate_mode, live, topk_idx + (int64_t)t * p.K,
+    const int sel = group_topk_gate<L, NPL>(key, p.K, p.gate_mode, live, topk_idx + (int64_t)t * p.K,
                                             topk_w + (int64_t)t * p.K);
-      if (cta_hist && live && sel >= 0) atomicAdd(&cta_hist[sel], 1);
-    }
+    if (cta_hist && live && sel >= 0) atomicAdd(&cta_hist[sel], 1);
   }
+}
+
+template <int L>
+__device__ __forceinline__ void select_rows_l(const RouteParams& p, const float* rows_smem, int rows, int t0,
+                                              int32_t* __restrict__ topk_idx, float* __restrict__ topk_w,
+                                              int32_t* cta_hist) {
+  const int per_lane = (p.E + L - 1) / L;        // experts per lane, rounded up to a power of two below
+#define MOEGPS_SEL(NPL) select_rows<L, NPL>(p, rows_smem, rows, t0, topk_idx, topk_w, cta_hist)
+  if (per_lane <= 1) MOEGPS_SEL(1);
+  else if (per_lane <= 2) MOEGPS_SEL(2);
+  else if (per_lane <= 4) MOEGPS_SEL(4);
+  else if (per_lane <= 8) MOEGPS_SEL(8);
+  else if (per_lane <= 16) MOEGPS_SEL(16);
+  else MOEGPS_SEL(32);                           // the launcher keeps E <= 32 * L
+#undef MOEGPS_SEL
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -124,13 +114,13 @@ route_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
              float* __restrict__ topk_w, float* __restrict__ logits_out, int32_t* __restrict__ hist,
              int32_t* __restrict__ status) {
   __shared__ int32_t cta_hist[256];       // this CTA's share of the histogram (used when hist != nullptr)
-  __shared__ float s_bias[256];           // fetched before the main loop so that the epilogue does not wait for it
+  __shared__ float s_bias[256];           // fetched while the stream runs
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  // [ ring (re-used as the partial-logit buffer) | barriers ]
+  // [ ring, later re-used as the partial-logit buffers | barriers ]
   const int part_bytes = BM * p.part_stride * 4;
   const int region0 = p.ring_bytes > part_bytes ? p.ring_bytes : part_bytes;
-  float* partial = reinterpret_cast<float*>(smem);
+  float* partial = reinterpret_cast<float*>(smem);       // [source slice][row of mine][part_stride]
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + region0);
   uint64_t* full = bars;                 // [stages]
   uint64_t* empty = bars + p.stages;     // [stages]
@@ -139,17 +129,16 @@ route_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t rank = cluster_ctarank();
+  const uint32_t rank = p.ks > 1 ? cluster_ctarank() : 0u;
   const int m0 = blockIdx.x * BM;
   const int nkb = (p.D + BK - 1) / BK;
   const int kb_begin = (int)rank * p.kb_per_cta;
   const int kb_end = min(nkb, kb_begin + p.kb_per_cta);
   const int stage_bytes = kABytes + p.e_pad * 128;
+  const int rows_per = BM / p.ks;
 
-  for (int e = threadIdx.x; e < p.E; e += kThreads) {
-    cta_hist[e] = 0;
-    s_bias[e] = bias ? bias[e] : 0.f;
-  }
+  // set-up: nothing here waits for global memory, so the stream starts within a few hundred cycles
+  if (threadIdx.x < 256) cta_hist[threadIdx.x] = 0;
   if (threadIdx.x == 0) {
     for (int i = 0; i < p.stages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
     mbar_init(acc_full, 1);
@@ -180,6 +169,8 @@ route_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         if (++stage == p.stages) { stage = 0; phase ^= 1u; }
       }
     }
+    __syncwarp();
+    if (p.ks > 1) { cluster_arrive_release(); cluster_wait_acquire(); }   // #1, see the drain warps
   } else if (warp == 1) {
     if (lane == 0) {
       const uint32_t idesc = idesc_bf16_f32(BM, p.e_pad);
@@ -200,65 +191,96 @@ route_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
       }
       if (ok && kb_begin < kb_end) mma_commit(acc_full);
     }
+    __syncwarp();
+    if (p.ks > 1) { cluster_arrive_release(); cluster_wait_acquire(); }   // #1
   } else if (warp < 6) {
-    // drain this CTA's partial logits: thread = token row, 32 columns per TMEM load
+    // drain: thread = token row of the tile.  The accumulator is complete once acc_full flips; from
+    // then on this CTA's ring is no longer read by its tensor core.
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
-    float* prow0 = partial + (size_t)row * p.part_stride;
-    if (kb_begin >= kb_end) {
-      // an empty K slice (only when D is short): its partial is zero
-      for (int c = 0; c < p.e_pad; ++c) prow0[c] = 0.f;
-    }
-    const bool ok = kb_begin < kb_end && mbar_wait(acc_full, 0, abort_flag);
+    const bool have = kb_begin < kb_end;          // an empty K slice (only when D is short) contributes zeros
+    const bool ok = (!have || mbar_wait(acc_full, 0, abort_flag)) && have;
     tc_fence_after_sync();
-    if (ok) {
-      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
-      float* prow = partial + (size_t)row * p.part_stride;
-      for (int c0 = 0; c0 < p.e_pad; c0 += 32) {
-        uint32_t v[32];
-        tmem_ld32(taddr + c0, v);
-        tmem_ld_wait();
-        // 16-byte stores: with a row stride of 4 (mod 8) words a quarter-warp covers all banks once
+    const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    if (p.ks > 1) cluster_arrive_release();       // #1: my tensor core has finished with my ring
+    const int owner = row / rows_per, row_local = row - owner * rows_per;
+    const uint32_t local = smem_u32(partial + ((size_t)rank * rows_per + row_local) * p.part_stride);
+    const uint32_t dst = p.ks > 1 ? map_to_cta(local, (uint32_t)owner) : local;
+    uint32_t cur[32];
+    if (ok) { tmem_ld32(taddr, cur); tmem_ld_wait(); }
+    if (p.ks > 1) cluster_wait_acquire();         // #1: every peer's ring is free as well
+    for (int c0 = 0; c0 < p.e_pad; c0 += 32) {
+      uint32_t nxt[32];
+      const bool more = c0 + 32 < p.e_pad;
+      if (more && ok) tmem_ld32(taddr + c0 + 32, nxt);      // overlaps the stores below
 #pragma unroll
-        for (int i = 0; i < 32; i += 4)
-          if (c0 + i < p.e_pad)
-            *reinterpret_cast<float4*>(prow + c0 + i) = make_float4(__uint_as_float(v[i]), __uint_as_float(v[i + 1]),
-                                                                    __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+      for (int i = 0; i < 32; i += 4) {
+        if (c0 + i < p.e_pad)
+          st_cluster_f32x4(dst + (uint32_t)(c0 + i) * 4u, ok ? __uint_as_float(cur[i]) : 0.f,
+                           ok ? __uint_as_float(cur[i + 1]) : 0.f, ok ? __uint_as_float(cur[i + 2]) : 0.f,
+                           ok ? __uint_as_float(cur[i + 3]) : 0.f);
+      }
+      if (more) {
+        if (ok) tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) cur[i] = nxt[i];
       }
     }
     tc_fence_before_sync();
+  } else {
+    // idle warps fetch the bias while the stream runs; it is read after the block barrier below
+    for (int e = threadIdx.x - 6 * 32; e < p.E; e += kThreads - 6 * 32) s_bias[e] = bias ? bias[e] : 0.f;
+    if (p.ks > 1) { cluster_arrive_release(); cluster_wait_acquire(); }   // #1
   }
   __syncwarp();
+  if (p.ks > 1) {
+    cluster_arrive_release();     // #2: my pushes are done ...
+    cluster_wait_acquire();       //     ... and so are everybody's into my shared memory
+  }
   __syncthreads();
   if (threadIdx.x == 0 && *abort_flag) {
     moegps_report(status, MOEGPS_ERR_TIMEOUT, (int)blockIdx.x);
     for (int i = 0; i < 1000; ++i) __nanosleep(1000);    // let copies still in flight land
   }
-  __syncwarp();
-  cluster_sync_all();           // every CTA's partial is complete and visible cluster-wide
 
-  // reduction + selection: CTA `rank` owns rows [rank*rows_per, (rank+1)*rows_per) of the tile
-  switch (p.ks) {
-    case 1: break;
-    case 2: reduce_partials<2>(p, partial, rank); break;
-    case 4: reduce_partials<4>(p, partial, rank); break;
-    default: reduce_partials<8>(p, partial, rank); break;
+  // The rows this CTA owns, tile rows [rank*rows_per, (rank+1)*rows_per): sum over the source slices
+  // in slice order, add the bias, 16 bytes per access, into slice 0's rows.
+  const int t0 = m0 + (int)rank * rows_per;
+  if (*abort_flag == 0) {
+    const int chunks = p.e_pad / 4;
+    const int slice_words = rows_per * p.part_stride;
+    for (int idx = threadIdx.x; idx < rows_per * chunks; idx += kThreads) {
+      const int r = idx / chunks, c = idx - r * chunks;
+      const int word = r * p.part_stride + 4 * c;
+      float4 s = *reinterpret_cast<const float4*>(partial + word);
+      for (int k = 1; k < p.ks; ++k) {
+        const float4 q = *reinterpret_cast<const float4*>(partial + (size_t)k * slice_words + word);
+        s.x += q.x; s.y += q.y; s.z += q.z; s.w += q.w;
+      }
+      const int e = 4 * c;       // (bias of padded experts: s_bias is read at e < 256 only; their keys are never used)
+      s.x += s_bias[e]; s.y += s_bias[e + 1]; s.z += s_bias[e + 2]; s.w += s_bias[e + 3];
+      *reinterpret_cast<float4*>(partial + word) = s;
+      if (logits_out && t0 + r < p.T) {
+        float* lo = logits_out + (int64_t)(t0 + r) * p.E;
+        if (e < p.E) lo[e] = s.x;
+        if (e + 1 < p.E) lo[e + 1] = s.y;
+        if (e + 2 < p.E) lo[e + 2] = s.z;
+        if (e + 3 < p.E) lo[e + 3] = s.w;
+      }
+    }
+    __syncthreads();
+    if (topk_idx) {
+      int32_t* const hc = hist ? cta_hist : nullptr;
+      switch (p.lanes) {
+        case 4: select_rows_l<4>(p, partial, rows_per, t0, topk_idx, topk_w, hc); break;
+        case 8: select_rows_l<8>(p, partial, rows_per, t0, topk_idx, topk_w, hc); break;
+        case 16: select_rows_l<16>(p, partial, rows_per, t0, topk_idx, topk_w, hc); break;
+        default: select_rows_l<32>(p, partial, rows_per, t0, topk_idx, topk_w, hc); break;
+      }
+    }
   }
   __syncthreads();
-  const int rows_per = BM / p.ks;
-  int32_t* const hc = hist ? cta_hist : nullptr;
-#define MOEGPS_ROUTE_SELECT(NPL) \
-  select_rows<NPL>(p, partial, (int)rank * rows_per, rows_per, m0, s_bias, topk_idx, topk_w, logits_out, hc);
-  if (p.E <= 8) { MOEGPS_ROUTE_SELECT(1) }               // experts per lane of an eight-lane group
-  else if (p.E <= 16) { MOEGPS_ROUTE_SELECT(2) }
-  else if (p.E <= 32) { MOEGPS_ROUTE_SELECT(4) }
-  else if (p.E <= 64) { MOEGPS_ROUTE_SELECT(8) }
-  else if (p.E <= 128) { MOEGPS_ROUTE_SELECT(16) }
-  else { MOEGPS_ROUTE_SELECT(32) }
-#undef MOEGPS_ROUTE_SELECT
-  __syncwarp();
-  cluster_sync_all();           // nobody leaves while a peer may still read its shared memory
-  if (hist) {                   // (the barrier above also orders this CTA's shared counters)
+  if (hist) {
     for (int e = threadIdx.x; e < p.E; e += kThreads) {
       const int c = cta_hist[e];
       if (c) atomicAdd(&hist[e], c);
@@ -295,6 +317,11 @@ int moegps_launch_route(moegps_ctx* ctx, const void* x, const void* wr, const fl
   while (p.tmem_cols < p.e_pad) p.tmem_cols *= 2;
   p.ring_bytes = p.stages * stage_bytes;
   p.part_stride = p.e_pad + 4;        // rows 16-byte aligned; 4 (mod 8) words apart: conflict-free 16-byte accesses
+  // lanes per token in the selection: the CTA's rows fill its threads in one pass where possible;
+  // at least K lanes (sub-lane k stores the k-th selection), at most 32 experts per lane
+  int lanes = 4;
+  while (lanes < 32 && (lanes * 2 * (BM / ks) <= kThreads || lanes < s.K || s.E > 32 * lanes)) lanes *= 2;
+  p.lanes = lanes;
   const int part_bytes = BM * p.part_stride * 4;
   const int region0 = p.ring_bytes > part_bytes ? p.ring_bytes : part_bytes;
   const size_t smem_bytes = 1024 + (size_t)region0 + (2 * p.stages + 1) * 8 + 64;

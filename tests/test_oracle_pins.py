@@ -272,6 +272,145 @@ def test_plan_bound_sandwich_and_monotone():
             prev = bound
 
 
+# ------------------------------------------------------------------------------ pack (Algorithm 1)
+def pack_invariants(n, home, cap, c_max, placed, share, load):
+    E, G = placed.shape
+    assert set(np.unique(placed)) <= {0, 1}
+    assert np.array_equal(share.sum(axis=1), n)                     # every token is served exactly once
+    assert (share >= 0).all() and ((share > 0) <= (placed == 1)).all()   # only by devices that host its expert
+    assert all(placed[e, home[e]] == 1 for e in range(E))           # the original copy is never removed
+    assert (placed.sum(axis=0) <= cap).all()                        # memory of every device respected
+    if c_max > 0:
+        assert (placed.sum(axis=1) <= c_max).all()
+    assert np.array_equal(load, share.sum(axis=0))
+
+
+def test_pack_paper_duplication_example():
+    with open(os.path.join(HERE, "golden", "duplication_example.txt")) as f:
+        line = [ln for ln in f if not ln.startswith("#")][0]
+    tokens, gpus, final = [part.split() for part in line.split("|")]
+    n, G = [int(v) for v in tokens], int(gpus[0])
+    placed, share, load, iters = oracle.pack(n, list(range(G)), [G] * G)
+    assert load.tolist() == [int(final[0])] * G                      # every GPU ends with the same load
+    assert placed[0].tolist() == [1] * G and placed[1:].sum() == 3   # only the popular expert is replicated
+    pack_invariants(np.array(n), list(range(G)), [G] * G, 0, placed, share, load)
+
+
+def test_pack_hand_worked_moves():
+    # ceil in Delta: loads (5, 0) -> Delta = 3 -> (2, 3); a floor would stop at (3, 2)
+    placed, share, load, iters = oracle.pack([5, 0], [0, 1], [2, 2])
+    assert load.tolist() == [2, 3] and iters == 1 and share.tolist() == [[2, 3], [0, 0]]
+    # ties: two hottest devices (0 and 1) and two coldest (2 and 3): device 0 gives to device 2 first
+    placed, share, load, iters = oracle.pack([4, 4, 0, 0], [0, 1, 2, 3], [2, 2, 2, 2])
+    assert share.tolist() == [[2, 0, 2, 0], [0, 2, 0, 2], [0, 0, 0, 0], [0, 0, 0, 0]] and iters == 2
+    # the biggest expert of the hottest device moves, and the lowest index among equally big ones
+    placed, share, load, iters = oracle.pack([3, 3, 1], [0, 0, 0], [3, 3], max_iters=1)
+    assert share.tolist() == [[0, 3], [3, 0], [1, 0]]                # Delta = ceil(7/2) = 4, but expert 0 has only 3
+    # nothing to do: one device, or loads already within one token
+    assert oracle.pack([7, 2], [0, 0], [2])[3] == 0
+    assert oracle.pack([3, 4], [0, 1], [2, 2])[3] == 0
+
+
+def test_pack_reaches_the_termination_target_when_unconstrained():
+    # with room everywhere and no copy cap every move is legal, so the loop can only end on its
+    # own condition: max L - min L <= 1, i.e. the optimum ceil(N / G)
+    for trial in range(40):
+        E, G = int(rng.integers(1, 20)), int(rng.integers(1, 9))
+        n = rng.integers(0, 200, size=E) * rng.integers(0, 2, size=E)
+        home = rng.integers(0, G, size=E)
+        placed, share, load, iters = oracle.pack(n, home, [E] * G)
+        assert load.max() - load.min() <= 1
+        assert load.max() == -(-int(n.sum()) // G)
+        pack_invariants(n, home, [E] * G, 0, placed, share, load)
+
+
+def optimal_max_load(n, home, cap, c_max):
+    """Brute force over every placement that keeps the original copies and respects memory and the
+    copy cap; for a fixed placement the best achievable max load is found by trying every way of
+    splitting every expert's tokens over its hosts (tiny inputs only)."""
+    import itertools
+    E, G = len(n), len(cap)
+    best = None
+    options = []
+    for e in range(E):
+        opts = []
+        for mask in range(1 << G):
+            if not (mask >> home[e]) & 1:
+                continue
+            if c_max > 0 and bin(mask).count("1") > c_max:
+                continue
+            opts.append(mask)
+        options.append(opts)
+    for masks in itertools.product(*options):
+        if any(sum((m >> g) & 1 for m in masks) > cap[g] for g in range(G)):
+            continue
+        splits = []
+        for e in range(E):
+            hosts = [g for g in range(G) if (masks[e] >> g) & 1]
+            ways = [w for w in itertools.product(range(n[e] + 1), repeat=len(hosts)) if sum(w) == n[e]]
+            splits.append([(hosts, w) for w in ways])
+        for combo in itertools.product(*splits):
+            load = [0] * G
+            for hosts, w in combo:
+                for g, k in zip(hosts, w):
+                    load[g] += k
+            m = max(load)
+            best = m if best is None or m < best else best
+    return best
+
+
+def test_pack_against_brute_force_on_tiny_inputs():
+    cases = 0
+    for trial in range(60):
+        E, G = int(rng.integers(1, 4)), int(rng.integers(1, 4))
+        n = [int(v) for v in rng.integers(0, 5, size=E)]
+        home = [int(v) for v in rng.integers(0, G, size=E)]
+        homed = [home.count(g) for g in range(G)]
+        cap = [homed[g] + int(rng.integers(0, 3)) for g in range(G)]
+        c_max = int(rng.integers(0, 3))
+        placed, share, load, iters = oracle.pack(n, home, cap, c_max)
+        pack_invariants(np.array(n), home, cap, c_max, placed, share, load)
+        opt = optimal_max_load(n, home, cap, c_max)
+        initial = max(sum(n[e] for e in range(E) if home[e] == g) for g in range(G))
+        assert opt <= load.max() <= initial          # a heuristic: never better than the optimum, never worse than doing nothing
+        if c_max == 0 and all(c >= E for c in cap):
+            assert load.max() == opt                 # unconstrained it is optimal
+        cases += 1
+    assert cases == 60
+
+
+def test_pack_respects_copy_cap_and_memory():
+    n = [1000, 10, 10, 10]
+    # c_max = 1: nothing may be copied, and a token can only go where its expert is: nothing moves
+    placed, share, load, iters = oracle.pack(n, [0, 1, 2, 3], [4] * 4, c_max=1)
+    assert iters == 0 and share.tolist() == np.diag(n).tolist()
+    # c_max = 2: the hot expert gets exactly one more copy
+    placed, share, load, iters = oracle.pack(n, [0, 1, 2, 3], [4] * 4, c_max=2)
+    assert placed[0].sum() == 2 and load.max() == 505
+    # no free place anywhere: same as no copies
+    placed, share, load, iters = oracle.pack(n, [0, 1, 2, 3], [1] * 4)
+    assert iters == 0 and placed.sum() == 4
+    with pytest.raises(ValueError):
+        oracle.pack(n, [0, 0, 0, 0], [3, 4, 4, 4])   # initial placement does not fit
+
+
+def test_pack_never_beats_the_slot_planner_bound():
+    # one replica per device (capacity 1, S = G devices, the experts on the first E): this is the
+    # setting of plan(), whose greedy is min-max optimal there: Algorithm 1 can match it, not beat it
+    for trial in range(20):
+        E, extra = int(rng.integers(1, 8)), int(rng.integers(0, 8))
+        n = rng.integers(0, 500, size=E)
+        G = E + extra
+        placed, share, load, iters = oracle.pack(n, list(range(E)), [1] * G)
+        _, _, _, bound = oracle.plan(n, G)
+        assert load.max() >= bound
+        pack_invariants(n, list(range(E)), [1] * G, 0, placed, share, load)
+    # one expert, three devices: 100 -> 50/50/0 -> 50/25/25 -> ... the loop keeps shifting tokens
+    # between the copies until the loads are within one token
+    placed, share, load, iters = oracle.pack([100], [0], [1, 1, 1])
+    assert sorted(load.tolist()) == [33, 33, 34] and iters > 2
+
+
 # ------------------------------------------------------------------------------ dispatch
 def closed_form_replica(i, n, r):
     return ((i + 1) * r - 1) // n
