@@ -86,7 +86,7 @@ def record_traffic(csv_path: str, workload: str, pairs: int):
     for r in csv.DictReader(lines):
         rows.append(r)
     out = {}
-    for key, tag in (("gate_up", "grouped_gemm_kernel<1>"), ("down", "grouped_gemm_kernel<0>")):
+    for key, tag in (("gate_up", "grouped_gemm_kernel<1,"), ("down", "grouped_gemm_kernel<0,")):
         acc = {"dram__bytes_read.sum": [], "dram__bytes_write.sum": []}
         for r in rows:
             if tag not in r.get("Kernel Name", ""):
@@ -202,11 +202,10 @@ def whole_job_rate(world: int, tokens_per_rank: int, steps: int, elapsed_ms: flo
 class Bench:
     """One workload resident on the device: layer, inputs, prediction."""
 
-    A = 128
-
     def __init__(self, w, rank: int, local_rank: int):
         from paper_2506_07366_b200 import binding
-        from paper_2506_07366_b200.layer import MoeLayer
+        from paper_2506_07366_b200.layer import MoeLayer, ROW_ALIGN
+        self.A = ROW_ALIGN
         self.w, self.dev = w, torch.device("cuda", local_rank)
         dev = self.dev
         self.shape = binding.Shape(w.T, w.D, w.F, w.E, w.K, w.S, w.gate_mode, self.A)
@@ -467,7 +466,7 @@ def run_ours(args):
     else:
         peak, peak_kind = peaks["bf16_burst"], " (burst bf16 GEMM: timed region < 2 s, boost clocks)"
     config = {"workload": w.name, "T": w.T, "D": w.D, "F": w.F, "E": w.E, "K": w.K, "S": w.S,
-              "row_align": Bench.A, "tokens_per_gpu": w.T, "prediction": w.prediction,
+              "row_align": b.A, "tokens_per_gpu": w.T, "prediction": w.prediction,
               "l2": "inputs larger than L2: %.2f GB of expert weights stream through it every step"
                     % (3 * w.E * w.D * w.F * 2 / 1e9)}
     config.update({k: stats[k] for k in ("skewness", "skewness_after_plan", "max_slot_load", "plan_bound",

@@ -232,6 +232,15 @@ MOEGPS_API int moegps_combine(moegps_ctx_t* ctx, const void* yp, const int32_t* 
 MOEGPS_API int moegps_predictor_update(moegps_ctx_t* ctx, const int32_t* hist, int64_t* state,
                                        int32_t* predicted_hist, void* stream);
 
+/* predictor_update_ema - the same estimate with geometric forgetting (Section 3.2.1 leaves the
+ * weights of its average over batches open; Section 3.1 discusses how often to predict and re-place):
+ * state holds per-expert counts in units of 2^-16 tokens and moves towards the new batch by
+ * floor((hist*2^16 - state) / 2^shift), i.e. a weight of 2^-shift for the newest batch (shift = 0: the
+ * last batch alone).  Integer arithmetic: exact and deterministic.  predicted_hist as above (state
+ * scaled down by a power of two to fit int32).  shift in [0,16]; state: int64 [E], zeroed to start. */
+MOEGPS_API int moegps_predictor_update_ema(moegps_ctx_t* ctx, const int32_t* hist, int64_t* state, int32_t shift,
+                                           int32_t* predicted_hist, void* stream);
+
 /* error_rate - the paper's quality metric of a predicted distribution (Section 3.2.1, with the
  * averaging of Section 3.3): mean over the experts of |p_est_e - p_e| / (1/E), where p_est and p are
  * predicted_hist and hist normalised to sum 1.  fp64, deterministic summation order.

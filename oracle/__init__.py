@@ -14,6 +14,7 @@ from .moe_oracle import (  # noqa: F401
     skewness,
     error_rate,
     predictor_update,
+    predictor_update_ema,
     plan,
     pack,
     replica_starts,

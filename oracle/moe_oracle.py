@@ -23,7 +23,7 @@ import numpy as np
 
 __all__ = [
     "bf16_bits_to_f64", "route_logits", "route", "histogram", "p_hat", "skewness", "error_rate",
-    "predictor_update",
+    "predictor_update", "predictor_update_ema",
     "plan", "pack", "replica_starts", "dispatch", "expert_ffn", "combine", "moe_layer",
 ]
 
@@ -148,6 +148,26 @@ def predictor_update(state, hist):
     while (max(s) >> shift) > 2 ** 31 - 1:
         shift += 1
     return s, np.array([v >> shift for v in s], dtype=np.int32)
+
+
+def predictor_update_ema(state, hist, shift: int):
+    """Exponentially weighted form of the same estimate (Section 3.2.1 speaks of a moving average
+    over batches without fixing its weights; the cumulative form above weights all batches alike,
+    this one forgets old batches geometrically with alpha = 2^-shift).  Integer arithmetic only:
+    the state holds per-expert counts in units of 2^-16 tokens and moves towards the new batch by
+    state += floor((hist * 2^16 - state) / 2^shift).  The prediction handed to the planner is the
+    state divided by the smallest power of two that makes its largest entry fit an int32 (only
+    proportions matter to the plan).  Returns (new_state as Python ints, predicted_hist int32)."""
+    if not (0 <= int(shift) <= 16):
+        raise ValueError("shift in 0..16")
+    h = [int(b) for b in np.asarray(hist).reshape(-1)]
+    if any(b < 0 for b in h):
+        raise ValueError("counts must be >= 0")
+    s = [int(a) + (((b << 16) - int(a)) >> int(shift)) for a, b in zip(np.asarray(state).reshape(-1), h)]
+    down = 0
+    while (max(s) >> down) > 2 ** 31 - 1:
+        down += 1
+    return s, np.array([v >> down for v in s], dtype=np.int32)
 
 
 # --------------------------------------------------------------------------------------------

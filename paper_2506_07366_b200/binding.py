@@ -56,7 +56,7 @@ EXPORTS = (
     "moegps_route_histogram", "moegps_route_logits", "moegps_histogram", "moegps_plan", "moegps_pack", "moegps_dispatch", "moegps_dispatch_static",
     "moegps_expert_ffn", "moegps_expert_ffn_gate_up", "moegps_expert_ffn_down", "moegps_combine",
     "moegps_status", "moegps_launch_count", "moegps_last_cuda_error", "moegps_error_string",
-    "moegps_selftest_bounded_wait", "moegps_predictor_update", "moegps_error_rate",
+    "moegps_selftest_bounded_wait", "moegps_predictor_update", "moegps_predictor_update_ema", "moegps_error_rate",
 )
 
 
@@ -107,6 +107,7 @@ def _lib():
         "moegps_combine": (ctypes.c_int, [vp] * 6),
         "moegps_selftest_bounded_wait": (ctypes.c_int, [vp, i64, vp]),
         "moegps_predictor_update": (ctypes.c_int, [vp] * 5),
+        "moegps_predictor_update_ema": (ctypes.c_int, [vp, vp, vp, i32, vp, vp]),
         "moegps_error_rate": (ctypes.c_int, [vp] * 5),
         "moegps_status": (ctypes.c_int, [vp, vp, _c_int32_p]),
         "moegps_launch_count": (i64, [vp]),
@@ -308,6 +309,13 @@ class Context:
             self._h, _ptr(hist, torch.int32, (s.E,), "hist"), _ptr(state, torch.int64, (s.E,), "state"),
             _ptr(predicted_hist, torch.int32, (s.E,), "predicted_hist"), _stream(stream)),
             "moegps_predictor_update")
+
+    def predictor_update_ema(self, hist, state, shift, predicted_hist, stream=None):
+        s = self.shape
+        self._check(_lib().moegps_predictor_update_ema(
+            self._h, _ptr(hist, torch.int32, (s.E,), "hist"), _ptr(state, torch.int64, (s.E,), "state"), int(shift),
+            _ptr(predicted_hist, torch.int32, (s.E,), "predicted_hist"), _stream(stream)),
+            "moegps_predictor_update_ema")
 
     def error_rate(self, predicted_hist, hist, error_rate, stream=None):
         s = self.shape

@@ -15,6 +15,11 @@
 // two smaller CTAs per SM (2-stage rings, one accumulator and 4 epilogue warps each), meant to let a
 // weight-streaming tile of a short slot overlap a tensor-bound tile of a long slot on one SM, was
 // measured 3-9 % slower on every workload (halving each ring costs more than the overlap returns).
+// Also measured and not kept: short slots (at most 128 rows) computed with swapped operands - the two
+// 128-row weight tiles of a stage as the MMAs' M, the slot's rows rounded up to 16 as N, transposed
+// epilogue - which cuts the tensor time of a 13-row slot eightfold.  Bit-exact, but the many-small-
+// expert layer it was meant for gained 2 % (its short slots are bound by streaming their weights,
+// not by the padded MMAs) while the bookkeeping cost the other layers 1-2 %.
 #include "common.cuh"
 #include "sm100.cuh"
 

@@ -36,6 +36,36 @@ predictor_update_kernel(const int32_t* __restrict__ hist, int E, long long* __re
   if (tid < E) predicted[tid] = (int32_t)(s >> shift);
 }
 
+// Exponentially weighted variant: the state holds counts in units of 2^-16 tokens and moves towards
+// the new batch by floor((hist * 2^16 - state) / 2^shift), i.e. alpha = 2^-shift.  Integer only.
+__global__ void __launch_bounds__(kThreads)
+predictor_update_ema_kernel(const int32_t* __restrict__ hist, int E, int shift, long long* __restrict__ state,
+                            int32_t* __restrict__ predicted, int32_t* __restrict__ status) {
+  __shared__ long long warp_max[kThreads / 32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  long long s = 0;
+  if (tid < E) {
+    int h = hist[tid];
+    if (h < 0) {
+      moegps_report(status, MOEGPS_ERR_BAD_INDEX, tid);
+      h = 0;
+    }
+    const long long old = state[tid];
+    s = old + ((((long long)h << 16) - old) >> shift);      // arithmetic shift = floor division
+    state[tid] = s;
+  }
+  long long m = s;
+#pragma unroll
+  for (int d = 16; d >= 1; d >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, d));
+  if (lane == 0) warp_max[warp] = m;
+  __syncthreads();
+  m = 0;
+  for (int w = 0; w < kThreads / 32; ++w) m = max(m, warp_max[w]);
+  int down = 0;
+  while ((m >> down) > 0x7fffffffll) ++down;
+  if (tid < E) predicted[tid] = (int32_t)(s >> down);
+}
+
 __global__ void __launch_bounds__(kThreads)
 error_rate_kernel(const int32_t* __restrict__ predicted, const int32_t* __restrict__ hist, int E,
                   double* __restrict__ out) {
@@ -78,6 +108,17 @@ extern "C" MOEGPS_API int moegps_predictor_update(moegps_ctx_t* ctx, const int32
   predictor_update_kernel<<<1, kThreads, 0, (cudaStream_t)stream>>>(hist, ctx->shape.E,
                                                                      reinterpret_cast<long long*>(state),
                                                                      predicted_hist, ctx->d_status);
+  MOEGPS_AFTER_LAUNCH(ctx);
+  return MOEGPS_OK;
+}
+
+extern "C" MOEGPS_API int moegps_predictor_update_ema(moegps_ctx_t* ctx, const int32_t* hist, int64_t* state,
+                                                      int32_t shift, int32_t* predicted_hist, void* stream) {
+  if (!ctx || !ok16(hist) || !ok16(state) || !ok16(predicted_hist) || shift < 0 || shift > 16)
+    return MOEGPS_ERR_INVALID_ARG;
+  if (int rc = moegps_check_device(ctx)) return rc;
+  predictor_update_ema_kernel<<<1, kThreads, 0, (cudaStream_t)stream>>>(
+      hist, ctx->shape.E, shift, reinterpret_cast<long long*>(state), predicted_hist, ctx->d_status);
   MOEGPS_AFTER_LAUNCH(ctx);
   return MOEGPS_OK;
 }

@@ -72,14 +72,14 @@ __device__ __forceinline__ void cluster_wait_acquire() {
 template <int L, int NPL>
 __device__ __forceinline__ void select_rows(const RouteParams& p, const float* rows_smem, int rows, int t0,
                                             int32_t* __restrict__ topk_idx, float* __restrict__ topk_w,
-                                            int32_t* cta_hist) {
+                                            int32_t* cta_hist, bool dry) {
   constexpr int kRowsPerWarp = 32 / L;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int sl = lane & (L - 1), grp = lane / L;
   for (int r0 = warp * kRowsPerWarp; r0 < rows; r0 += (kThreads / 32) * kRowsPerWarp) {   // rows % 8 == 0
     const int row = r0 + grp;
     const int t = t0 + row;
-    const bool live = t < p.T;
+    const bool live = t < p.T && !dry;
     const float* prow = rows_smem + (size_t)row * p.part_stride;
     uint32_t key[NPL];
 #pragma unroll
@@ -96,9 +96,9 @@ __device__ __forceinline__ void select_rows(const RouteParams& p, const float* r
 template <int L>
 __device__ __forceinline__ void select_rows_l(const RouteParams& p, const float* rows_smem, int rows, int t0,
                                               int32_t* __restrict__ topk_idx, float* __restrict__ topk_w,
-                                              int32_t* cta_hist) {
+                                              int32_t* cta_hist, bool dry) {
   const int per_lane = (p.E + L - 1) / L;        // experts per lane, rounded up to a power of two below
-#define MOEGPS_SEL(NPL) select_rows<L, NPL>(p, rows_smem, rows, t0, topk_idx, topk_w, cta_hist)
+#define MOEGPS_SEL(NPL) select_rows<L, NPL>(p, rows_smem, rows, t0, topk_idx, topk_w, cta_hist, dry)
   if (per_lane <= 1) MOEGPS_SEL(1);
   else if (per_lane <= 2) MOEGPS_SEL(2);
   else if (per_lane <= 4) MOEGPS_SEL(4);
@@ -106,6 +106,23 @@ __device__ __forceinline__ void select_rows_l(const RouteParams& p, const float*
   else if (per_lane <= 16) MOEGPS_SEL(16);
   else MOEGPS_SEL(32);                           // the launcher keeps E <= 32 * L
 #undef MOEGPS_SEL
+}
+
+// The selection stage, deliberately NOT inlined: it is called twice from the kernel - first by the
+// warps that have nothing to do while the tile streams, as a dry run (`dry`: garbage rows, nothing
+// stored, nothing counted) whose only purpose is to pull this code into the SM's instruction cache,
+// then by all warps for real.  The kernel runs once per layer, right after GEMMs that have flushed
+// every cache, and without the dry run a large share of the selection phase is spent waiting for
+// instruction fetches (the profiler's no_instruction stall was the largest single reason).
+__device__ __noinline__ void select_stage(const RouteParams& p, const float* rows_smem, int rows, int t0,
+                                          int32_t* __restrict__ topk_idx, float* __restrict__ topk_w,
+                                          int32_t* cta_hist, bool dry) {
+  switch (p.lanes) {
+    case 4: select_rows_l<4>(p, rows_smem, rows, t0, topk_idx, topk_w, cta_hist, dry); break;
+    case 8: select_rows_l<8>(p, rows_smem, rows, t0, topk_idx, topk_w, cta_hist, dry); break;
+    case 16: select_rows_l<16>(p, rows_smem, rows, t0, topk_idx, topk_w, cta_hist, dry); break;
+    default: select_rows_l<32>(p, rows_smem, rows, t0, topk_idx, topk_w, cta_hist, dry); break;
+  }
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -230,6 +247,7 @@ route_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
   } else {
     // idle warps fetch the bias while the stream runs; it is read after the block barrier below
     for (int e = threadIdx.x - 6 * 32; e < p.E; e += kThreads - 6 * 32) s_bias[e] = bias ? bias[e] : 0.f;
+    if (topk_idx) select_stage(p, partial, rows_per, m0, topk_idx, topk_w, nullptr, true);   // warms the instruction cache
     if (p.ks > 1) { cluster_arrive_release(); cluster_wait_acquire(); }   // #1
   }
   __syncwarp();
@@ -269,15 +287,7 @@ route_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
       }
     }
     __syncthreads();
-    if (topk_idx) {
-      int32_t* const hc = hist ? cta_hist : nullptr;
-      switch (p.lanes) {
-        case 4: select_rows_l<4>(p, partial, rows_per, t0, topk_idx, topk_w, hc); break;
-        case 8: select_rows_l<8>(p, partial, rows_per, t0, topk_idx, topk_w, hc); break;
-        case 16: select_rows_l<16>(p, partial, rows_per, t0, topk_idx, topk_w, hc); break;
-        default: select_rows_l<32>(p, partial, rows_per, t0, topk_idx, topk_w, hc); break;
-      }
-    }
+    if (topk_idx) select_stage(p, partial, rows_per, t0, topk_idx, topk_w, hist ? cta_hist : nullptr, false);
   }
   __syncthreads();
   if (hist) {

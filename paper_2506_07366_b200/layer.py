@@ -9,6 +9,12 @@ import torch
 
 from .binding import Context, Shape, workspace_bytes
 
+# Row alignment of the slot buckets that the benchmark and the serving examples use: slot starts are
+# multiples of 16 rows.  The grouped GEMM accepts any alignment (its tiles start at the slot's first
+# row and only rows of the slot are written); a small one keeps the permuted buffers compact - with
+# 288 slots, 128-row alignment would pad 32768 pairs to about 56000 rows, 16-row alignment to 35000.
+ROW_ALIGN = 16
+
 
 class MoeLayer:
     def __init__(self, shape: Shape, w_router, bias, w_gate, w_up, w_down, device=None):
@@ -58,6 +64,34 @@ class MoeLayer:
         c.expert_ffn(self.xp, self.slot_row_off, self.slot_expert, self.w_gate, self.w_up,
                      self.w_down, self.h_ws, self.yp, stream)
         c.combine(self.yp, self.pair_row, self.topk_w, out, stream)
+        return out
+
+    def start_prediction(self, replan_every: int = 1, ema_shift: int | None = None):
+        """Distribution-Only Prediction in a loop (paper, Sections 3.1 and 3.2.1): from now on
+        forward_predicted() feeds every batch's histogram to the predictor state and renews the
+        plan from the prediction after every `replan_every`-th batch (the paper's prediction and
+        placement frequency).  `ema_shift` = None keeps cumulative counts (every batch weighs the
+        same); an integer k forgets old batches with weight 2^-k for the newest one.  The first
+        batches run under the plan of an all-zero prediction (the spare slots spread evenly)."""
+        if replan_every < 1:
+            raise ValueError("replan_every >= 1")
+        self._every, self._ema_shift, self._batches = int(replan_every), ema_shift, 0
+        self._state = torch.zeros(self.shape.E, dtype=torch.int64, device=self.w_router.device)
+        self.pred.zero_()
+        self.ctx.plan(self.pred, self.shape.S, self.replicas, self.slot_off, self.slot_expert, self.bound)
+        self._planned = True
+
+    def forward_predicted(self, x, stream=None, out=None):
+        """forward() under the current plan, then predictor update (and re-plan when due)."""
+        out = self.forward(x, stream, out)
+        if self._ema_shift is None:
+            self.ctx.predictor_update(self.hist, self._state, self.pred, stream)
+        else:
+            self.ctx.predictor_update_ema(self.hist, self._state, self._ema_shift, self.pred, stream)
+        self._batches += 1
+        if self._batches % self._every == 0:
+            self.ctx.plan(self.pred, self.shape.S, self.replicas, self.slot_off, self.slot_expert, self.bound,
+                          stream)
         return out
 
     def capture(self, x, predicted_hist=None):

@@ -12,7 +12,7 @@ import torch
 
 import oracle
 from paper_2506_07366_b200 import binding, workloads as wl
-from paper_2506_07366_b200.layer import MoeLayer
+from paper_2506_07366_b200.layer import MoeLayer, ROW_ALIGN
 from tests import harness as hz
 
 pytestmark = pytest.mark.gpu
@@ -130,7 +130,7 @@ class ExpertsOnDemand:
 
 # name -> how the float outputs are compared at full size:
 #   "all"   every occupied row of yp and every token of out (the oracle needs seconds for these)
-#   "tiles" the first and the last occupied row of EVERY 128-row tile of every slot for yp - so a
+#   "tiles" the first and the last occupied row of EVERY 128-row stretch of every slot for yp - so a
 #           defect confined to one row tile, one slot or one round of the persistent tile loop shows -
 #           and out on the tokens that own a seeded subset of those rows
 FULL = [("mixtral", "all"), ("mixtral_skew", "tiles"), ("many_expert", "all"), ("fine_grained", "tiles")]
@@ -150,7 +150,7 @@ def test_layer_full_size(name, coverage):
     ref_idx, ref_w, ref_logits = oracle.route(xb, wrb, bb, w.K, w.gate_mode)
     ref_hist = oracle.histogram(ref_idx, w.E)
     pred = hz.predicted_histogram(w, ref_hist, wr.cpu(), bias.cpu())
-    A = 128
+    A = ROW_ALIGN                                   # the launch configuration the benchmark times
     rep, so, se, bound = oracle.plan(pred, w.S)
     sro, rp, pr, _ = oracle.dispatch(None, ref_idx, ref_hist, rep, so, w.S, A)
 
@@ -193,8 +193,8 @@ def test_layer_full_size(name, coverage):
         picked = []
         for s in range(w.S):
             n_occ = int(np.count_nonzero(rp[sro[s]:sro[s + 1]] >= 0))       # occupied rows lead the slot
-            for lo in range(0, n_occ, A):
-                picked += [sro[s] + lo, sro[s] + min(lo + A, n_occ) - 1]
+            for lo in range(0, n_occ, 128):
+                picked += [sro[s] + lo, sro[s] + min(lo + 128, n_occ) - 1]
         yp_rows = np.unique(np.array(picked, dtype=np.int64))
         assert (rp[yp_rows] >= 0).all()
         rng = np.random.default_rng(w.seed)
@@ -223,3 +223,8 @@ def test_plan_study_runs_on_a_small_workload():
         assert r["max_slot_load"] == r["plan_bound"]          # exact prediction: the split realises the plan
         assert r["prediction_error_rate"] == 0.0
         assert r["ffn_ms_bottleneck"] > 0 and r["ffn_ms_even_share"] > 0
+        assert r["ffn_ms_whole_layer_one_device"] > 0
+    # a copy cap of 2 (Algorithm 1's C_max) leaves slots empty once every expert worth copying has two
+    capped = plan_study.study("tiny", extras=[12], noises=[0.0], c_maxes=[0, 2], in_situ=False)
+    assert capped[0]["slots_used"] == 20 and capped[1]["slots_used"] == 16
+    assert capped[1]["max_slot_load"] >= capped[0]["max_slot_load"]

@@ -95,3 +95,51 @@ def test_closed_loop_histogram_predictor_plan():
         ctx.check_status()
         assert np.array_equal(pred.cpu().numpy(), ref_pred)
     assert all(0.0 <= e < 0.5 for e in errors) and errors[-1] <= errors[0] + 0.05
+
+
+@pytest.mark.parametrize("E,shift", [(1, 0), (8, 1), (64, 3), (256, 6), (200, 16)])
+def test_predictor_update_ema_matches_oracle_over_batches(E, shift):
+    rng = np.random.default_rng(7 * E + shift)
+    ctx = binding.Context(binding.Shape(8, 64, 64, E, 1, E, 0, 1))
+    state = torch.zeros(E, dtype=torch.int64, device=DEV)
+    pred = torch.full((E,), -7, dtype=torch.int32, device=DEV)
+    ref_state = [0] * E
+    for b in range(8):
+        hist = rng.integers(0, 2 ** 31 - 1 if b == 3 else 60000, size=E)     # one batch of huge counts: the scaling path
+        hist[rng.random(E) < 0.2] = 0
+        ctx.predictor_update_ema(i32(hist), state, shift, pred)
+        ref_state, ref_pred = oracle.predictor_update_ema(ref_state, hist, shift)
+        ctx.check_status()
+        assert state.cpu().tolist() == ref_state
+        assert np.array_equal(pred.cpu().numpy(), ref_pred)
+    with pytest.raises(binding.MoegpsError):
+        ctx.predictor_update_ema(i32(hist), state, 17, pred)
+
+
+def test_layer_replans_every_n_batches_from_the_predictor():
+    """The loop of Section 3.1 with a chosen prediction / placement frequency: every batch updates the
+    predictor state from its own histogram; every n-th batch the plan is renewed from the prediction."""
+    from paper_2506_07366_b200 import workloads as wl
+    from paper_2506_07366_b200.layer import MoeLayer
+    w = wl.WORKLOADS["tiny"].scaled(S=12)
+    wr, bias = wl.router(w, DEV)
+    w1, w3, w2 = wl.expert_weights(w, DEV)
+    shape = binding.Shape(w.T, w.D, w.F, w.E, w.K, w.S, w.gate_mode, 128)
+    for every, shift in ((1, None), (3, None), (2, 2)):
+        layer = MoeLayer(shape, wr, bias, w1, w3, w2)
+        layer.start_prediction(replan_every=every, ema_shift=shift)
+        ref_state, ref_pred = [0] * w.E, np.zeros(w.E, dtype=np.int32)
+        ref_rep = oracle.plan(ref_pred, w.S)[0]
+        for b in range(7):
+            x = wl.activations(w.scaled(number=w.number + 11 * b), DEV)
+            assert np.array_equal(layer.replicas.cpu().numpy(), ref_rep), (every, shift, b)   # the plan batch b runs under
+            layer.forward_predicted(x)
+            layer.ctx.check_status()
+            hist = layer.hist.cpu().numpy()
+            if shift is None:
+                ref_state, ref_pred = oracle.predictor_update(ref_state, hist)
+            else:
+                ref_state, ref_pred = oracle.predictor_update_ema(ref_state, hist, shift)
+            if (b + 1) % every == 0:
+                ref_rep = oracle.plan(ref_pred, w.S)[0]
+        assert np.array_equal(layer.replicas.cpu().numpy(), ref_rep)

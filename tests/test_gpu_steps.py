@@ -269,6 +269,13 @@ FFN_CASES = [
     (12288, 1024, 1024, 8, 2, 8, 128, 0.8),
     (12288, 1024, 1024, 8, 2, 12, 1, 0.8),     # the same with unaligned slots and replicas
     (6000, 2048, 256, 4, 2, 6, 128, 1.0),      # down GEMM with 8 column tiles per row tile, 32 K-blocks in gate+up
+    # a mix of short (under 128 rows) and long slots at small row alignments, ragged weight tails (F, D not
+    # multiples of 128): tiles of short slots read into the following slots' rows and must not write there
+    (900, 256, 384, 64, 4, 80, 16, 1.2),
+    (900, 256, 384, 64, 4, 80, 1, 1.2),        # extents that are not multiples of 16: the tile reads into the next slot
+    (700, 200, 328, 24, 3, 30, 8, 0.7),
+    (130, 512, 640, 3, 1, 3, 16, 0.0),         # extents of 48, 48, 48 ... and single slots just below / above 128 rows
+    (257, 128, 128, 2, 1, 2, 1, 0.0),
 ]
 
 

@@ -644,3 +644,40 @@ def test_predictor_scales_huge_counts_by_a_power_of_two():
     assert pred.tolist() == [2 ** 31 - 1, 5]               # still fits: no scaling
     with pytest.raises(ValueError):
         oracle.predictor_update([1, 1], [0, -1])
+
+
+def test_predictor_ema_special_cases_and_closed_form():
+    from fractions import Fraction
+    # alpha = 1 (shift 0): the state is the last batch, in units of 2^-16 tokens
+    state, pred = oracle.predictor_update_ema([123456, 7], [10, 20], 0)
+    assert state == [10 << 16, 20 << 16]
+    # a constant input is a fixed point, whatever the weight
+    for shift in (1, 3, 8, 16):
+        state, _ = oracle.predictor_update_ema([5 << 16, 0, 777 << 16], [5, 0, 777], shift)
+        assert state == [5 << 16, 0, 777 << 16]
+    # against the exact recurrence s_t = s_{t-1} + (h_t 2^16 - s_{t-1}) / 2^k in rationals: every step
+    # floors once, and the error it leaves decays like the state does, so the two stay within 2^k units
+    seq = rng.integers(0, 100000, size=(40, 6))
+    for shift in (1, 2, 5):
+        state, exact = [0] * 6, [Fraction(0)] * 6
+        for h in seq:
+            state, pred = oracle.predictor_update_ema(state, h, shift)
+            exact = [x + (Fraction(int(v) << 16) - x) / 2 ** shift for x, v in zip(exact, h)]
+            assert all(0 <= float(x - s) <= 2 ** shift for x, s in zip(exact, state))
+        # the textbook form: a geometrically weighted sum of the inputs
+        a = Fraction(1, 2 ** shift)
+        closed = [sum(a * (1 - a) ** (len(seq) - 1 - i) * (int(seq[i][e]) << 16) for i in range(len(seq))) for e in range(6)]
+        assert all(abs(float(c - x)) < 1e-6 for c, x in zip(closed, exact))
+    # proportions: two experts fed in the ratio 3:1 are predicted in that ratio
+    state = [0, 0]
+    for _ in range(200):
+        state, pred = oracle.predictor_update_ema(state, [3000, 1000], 4)
+    assert abs(pred[0] / pred[1] - 3.0) < 1e-3
+    # a step in the input is followed monotonically, and old batches are forgotten (unlike the cumulative form)
+    state, seen = [1000 << 16], []
+    for _ in range(60):
+        state, pred = oracle.predictor_update_ema(state, [0], 2)
+        seen.append(state[0])
+    assert seen == sorted(seen, reverse=True) and seen[-1] < (1 << 16) // 100
+    with pytest.raises(ValueError):
+        oracle.predictor_update_ema([0], [1], 17)
