@@ -20,6 +20,9 @@
 // epilogue - which cuts the tensor time of a 13-row slot eightfold.  Bit-exact, but the many-small-
 // expert layer it was meant for gained 2 % (its short slots are bound by streaming their weights,
 // not by the padded MMAs) while the bookkeeping cost the other layers 1-2 %.
+// And: cutting the tiles of a last round that is at most half full into two 128-column halves (down
+// GEMM; 7.35 rounds of tiles on the Mixtral-shaped layer) gained 1 % there and nothing elsewhere, so
+// the partial last round is not what separates the down GEMM from the gate+up GEMM.
 #include "common.cuh"
 #include "sm100.cuh"
 
