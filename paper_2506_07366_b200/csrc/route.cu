@@ -108,6 +108,37 @@ __device__ __forceinline__ void select_rows_l(const RouteParams& p, const float*
 #undef MOEGPS_SEL
 }
 
+// Sum of the KS partial logits of the rows this CTA owns, in slice order, plus the bias, 16 bytes per
+// access, into slice 0's rows (and to logits_out for the debug entry point).  Not inlined for the
+// same reason as select_stage below: idle warps run it once as a dry run (`dry`: nothing is stored)
+// while the tile streams, which brings its code into the instruction cache.
+__device__ __noinline__ void reduce_stage(const RouteParams& p, float* partial, const float* s_bias, int rows_per,
+                                          int t0, float* __restrict__ logits_out, bool dry) {
+  const int chunks = p.e_pad / 4;
+  const int slice_words = rows_per * p.part_stride;
+  // (the dry run is made by warps 6 and up: they start at the first items so that the body is executed)
+  for (int idx = dry ? (int)threadIdx.x - 6 * 32 : (int)threadIdx.x; idx < rows_per * chunks; idx += kThreads) {
+    const int r = idx / chunks, c = idx - r * chunks;
+    const int word = r * p.part_stride + 4 * c;
+    float4 s = *reinterpret_cast<const float4*>(partial + word);
+    for (int k = 1; k < p.ks; ++k) {
+      const float4 q = *reinterpret_cast<const float4*>(partial + (size_t)k * slice_words + word);
+      s.x += q.x; s.y += q.y; s.z += q.z; s.w += q.w;
+    }
+    const int e = 4 * c;         // (bias of padded experts: s_bias is read below 256 only; their keys are never used)
+    s.x += s_bias[e]; s.y += s_bias[e + 1]; s.z += s_bias[e + 2]; s.w += s_bias[e + 3];
+    if (dry) continue;
+    *reinterpret_cast<float4*>(partial + word) = s;
+    if (logits_out && t0 + r < p.T) {
+      float* lo = logits_out + (int64_t)(t0 + r) * p.E;
+      if (e < p.E) lo[e] = s.x;
+      if (e + 1 < p.E) lo[e + 1] = s.y;
+      if (e + 2 < p.E) lo[e + 2] = s.z;
+      if (e + 3 < p.E) lo[e + 3] = s.w;
+    }
+  }
+}
+
 // The selection stage, deliberately NOT inlined: it is called twice from the kernel - first by the
 // warps that have nothing to do while the tile streams, as a dry run (`dry`: garbage rows, nothing
 // stored, nothing counted) whose only purpose is to pull this code into the SM's instruction cache,
@@ -247,7 +278,8 @@ route_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
   } else {
     // idle warps fetch the bias while the stream runs; it is read after the block barrier below
     for (int e = threadIdx.x - 6 * 32; e < p.E; e += kThreads - 6 * 32) s_bias[e] = bias ? bias[e] : 0.f;
-    if (topk_idx) select_stage(p, partial, rows_per, m0, topk_idx, topk_w, nullptr, true);   // warms the instruction cache
+    reduce_stage(p, partial, s_bias, rows_per, m0, nullptr, true);                            // both warm the
+    if (topk_idx) select_stage(p, partial, rows_per, m0, topk_idx, topk_w, nullptr, true);   // instruction cache
     if (p.ks > 1) { cluster_arrive_release(); cluster_wait_acquire(); }   // #1
   }
   __syncwarp();
@@ -265,27 +297,7 @@ route_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
   // in slice order, add the bias, 16 bytes per access, into slice 0's rows.
   const int t0 = m0 + (int)rank * rows_per;
   if (*abort_flag == 0) {
-    const int chunks = p.e_pad / 4;
-    const int slice_words = rows_per * p.part_stride;
-    for (int idx = threadIdx.x; idx < rows_per * chunks; idx += kThreads) {
-      const int r = idx / chunks, c = idx - r * chunks;
-      const int word = r * p.part_stride + 4 * c;
-      float4 s = *reinterpret_cast<const float4*>(partial + word);
-      for (int k = 1; k < p.ks; ++k) {
-        const float4 q = *reinterpret_cast<const float4*>(partial + (size_t)k * slice_words + word);
-        s.x += q.x; s.y += q.y; s.z += q.z; s.w += q.w;
-      }
-      const int e = 4 * c;       // (bias of padded experts: s_bias is read at e < 256 only; their keys are never used)
-      s.x += s_bias[e]; s.y += s_bias[e + 1]; s.z += s_bias[e + 2]; s.w += s_bias[e + 3];
-      *reinterpret_cast<float4*>(partial + word) = s;
-      if (logits_out && t0 + r < p.T) {
-        float* lo = logits_out + (int64_t)(t0 + r) * p.E;
-        if (e < p.E) lo[e] = s.x;
-        if (e + 1 < p.E) lo[e + 1] = s.y;
-        if (e + 2 < p.E) lo[e + 2] = s.z;
-        if (e + 3 < p.E) lo[e + 3] = s.w;
-      }
-    }
+    reduce_stage(p, partial, s_bias, rows_per, t0, logits_out, false);
     __syncthreads();
     if (topk_idx) select_stage(p, partial, rows_per, t0, topk_idx, topk_w, hist ? cta_hist : nullptr, false);
   }
