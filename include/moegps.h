@@ -148,6 +148,17 @@ MOEGPS_API int moegps_pack(moegps_ctx_t* ctx, const int32_t* predicted_hist, con
                            const int32_t* capacity, int32_t n_devices, int32_t* placement, int32_t* share,
                            int32_t* load, int32_t* iterations, void* stream);
 
+/* pack_slots - the placement of moegps_pack as the slot tables the rest of the path works on: one
+ * slot per (expert, device) copy, experts in ascending order and, within an expert, its devices in
+ * ascending order; slot_share[s] = the predicted tokens Algorithm 1's dispatch gave that copy,
+ * slot_device[s] = its device; slots beyond the last copy are empty (expert -1, device -1, share 0).
+ * placement, share: int32 [E,G] from moegps_pack; n_devices = G.
+ * replicas: int32 [E]; slot_off: int32 [E+1]; slot_expert, slot_share, slot_device: int32 [S].
+ * More copies than shape.S slots are reported as MOEGPS_ERR_BAD_INDEX (the surplus is not written). */
+MOEGPS_API int moegps_pack_slots(moegps_ctx_t* ctx, const int32_t* placement, const int32_t* share,
+                                 int32_t n_devices, int32_t* replicas, int32_t* slot_off, int32_t* slot_expert,
+                                 int32_t* slot_share, int32_t* slot_device, void* stream);
+
 /* dispatch - the routing shuffle (paper, Section 2 all-to-all; Algorithm 1's dispatch d and its
  * "first tokens" rule): pairs of expert e, in flat pair order, are split into r_e contiguous
  * balanced ranges (replica rho takes stable ranks floor(rho*n_e/r_e) .. floor((rho+1)*n_e/r_e)-1)
@@ -164,6 +175,18 @@ MOEGPS_API int moegps_dispatch(moegps_ctx_t* ctx, const void* x, const int32_t* 
                     const int32_t* replicas, const int32_t* slot_off,
                     int32_t* slot_row_off, int32_t* row_pair, int32_t* pair_row,
                     void* xp, void* workspace, void* stream);
+
+/* dispatch_shares - moegps_dispatch for a placement made by moegps_pack / moegps_pack_slots (paper,
+ * Algorithm 1: the dispatch d sends different numbers of an expert's tokens to its copies).  The
+ * copies of expert e take shares of its ACTUAL pairs in proportion to slot_share (the predicted
+ * tokens each copy was given): copy rho takes the stable ranks floor(n_e c_rho / c) ..
+ * floor(n_e c_{rho+1} / c) - 1, c_rho = the shares of the copies before it, c their sum; an expert
+ * whose shares are all zero (the prediction gave it nothing) is split evenly as in moegps_dispatch.
+ * slot_share: int32 [S] >= 0, at most 2^31-1 per expert in total.  Everything else as moegps_dispatch. */
+MOEGPS_API int moegps_dispatch_shares(moegps_ctx_t* ctx, const void* x, const int32_t* topk_idx,
+                                      const int32_t* hist, const int32_t* replicas, const int32_t* slot_off,
+                                      const int32_t* slot_share, int32_t* slot_row_off, int32_t* row_pair,
+                                      int32_t* pair_row, void* xp, void* workspace, void* stream);
 
 /* dispatch_static - moegps_dispatch without the `workspace` argument.  (The paper has no
  * counterpart: this is a deployment convenience, not a step of the method.)

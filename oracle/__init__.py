@@ -17,7 +17,9 @@ from .moe_oracle import (  # noqa: F401
     predictor_update_ema,
     plan,
     pack,
+    pack_slots,
     replica_starts,
+    replica_starts_by_share,
     dispatch,
     expert_ffn,
     combine,

@@ -24,7 +24,8 @@ import numpy as np
 __all__ = [
     "bf16_bits_to_f64", "route_logits", "route", "histogram", "p_hat", "skewness", "error_rate",
     "predictor_update", "predictor_update_ema",
-    "plan", "pack", "replica_starts", "dispatch", "expert_ffn", "combine", "moe_layer",
+    "plan", "pack", "pack_slots", "replica_starts", "replica_starts_by_share", "dispatch", "expert_ffn",
+    "combine", "moe_layer",
 ]
 
 
@@ -298,6 +299,32 @@ def pack(pred_hist, home, capacity, c_max: int = 0, max_iters: int = 1 << 20):
             np.array(load, dtype=np.int64), iters)
 
 
+def pack_slots(placement, share, S: int):
+    """The placement of Algorithm 1 as slot tables: one slot per (expert, device) copy, experts in
+    ascending order and, within an expert, its devices in ascending order (the numbering dispatch
+    expects: expert e owns slots slot_off[e] .. slot_off[e+1]-1).  slot_share[s] is the number of
+    predicted tokens the algorithm's dispatch d assigned to that copy, slot_device[s] its device;
+    slots beyond the last copy are empty (expert -1, device -1, share 0).
+    Returns (replicas [E], slot_off [E+1], slot_expert [S], slot_share [S], slot_device [S])."""
+    P = np.asarray(placement)
+    sh = np.asarray(share)
+    E, G = P.shape
+    replicas = [int(P[e].sum()) for e in range(E)]
+    if sum(replicas) > S:
+        raise ValueError("more copies than slots")
+    slot_off = [0] * (E + 1)
+    slot_expert, slot_share, slot_device = [-1] * S, [0] * S, [-1] * S
+    for e in range(E):
+        slot_off[e + 1] = slot_off[e] + replicas[e]
+        s = slot_off[e]
+        for g in range(G):
+            if P[e][g]:
+                slot_expert[s], slot_share[s], slot_device[s] = e, int(sh[e][g]), g
+                s += 1
+    as_i32 = lambda v: np.array(v, dtype=np.int32)  # noqa: E731
+    return as_i32(replicas), as_i32(slot_off), as_i32(slot_expert), as_i32(slot_share), as_i32(slot_device)
+
+
 # --------------------------------------------------------------------------------------------
 # dispatch  (the routing all-to-all of Section 2 on one device; replica choice of Algorithm 1)
 # --------------------------------------------------------------------------------------------
@@ -307,7 +334,24 @@ def replica_starts(n_e: int, r_e: int):
     return [(rho * n_e) // r_e for rho in range(r_e + 1)]
 
 
-def dispatch(x, topk_idx, hist, replicas, slot_off, S: int, row_align: int = 1):
+def replica_starts_by_share(n_e: int, shares):
+    """Split of an expert's n_e ACTUAL pairs over its copies in proportion to the predicted tokens
+    that Algorithm 1's dispatch gave each copy: copy rho takes the stable ranks
+    start[rho] .. start[rho+1]-1 with start[rho] = floor(n_e * (shares[0] + .. + shares[rho-1]) / sum).
+    Every copy's load is within one pair of its proportional part.  When the prediction gave the
+    expert no tokens at all (sum = 0) nothing is known and the split is the balanced one."""
+    sh = [int(v) for v in shares]
+    tot = sum(sh)
+    if tot <= 0:
+        return replica_starts(n_e, len(sh))
+    cum, out = 0, [0]
+    for v in sh:
+        cum += v
+        out.append((n_e * cum) // tot)
+    return out
+
+
+def dispatch(x, topk_idx, hist, replicas, slot_off, S: int, row_align: int = 1, slot_share=None):
     """Lossless, stable permutation of routed pairs into slot buckets.
 
     For pair p (expert e = topk_idx[p]) the stable rank is i_p = #{q < p : topk_idx[q] = e}
@@ -315,6 +359,9 @@ def dispatch(x, topk_idx, hist, replicas, slot_off, S: int, row_align: int = 1):
     rho whose rank range contains i_p, i.e. slot s = slot_off[e] + rho, at row
     slot_row_off[s] + (i_p - start[rho]).  Slot s begins at a multiple of `row_align`;
     slot_row_off[s+1] = round_up(slot_row_off[s] + load_s, row_align).
+
+    With `slot_share` (int [S], from pack_slots) the copies of an expert take shares of its pairs in
+    proportion to those predicted counts instead of equal shares (replica_starts_by_share).
 
     Returns (slot_row_off int32 [S+1], row_pair int32 [Rcap] with -1 on padding rows,
              pair_row int32 [R], Xp [Rcap, D] bit copies of the token rows (zeros on padding)),
@@ -340,7 +387,10 @@ def dispatch(x, topk_idx, hist, replicas, slot_off, S: int, row_align: int = 1):
     load = [0] * S
     starts = []
     for e in range(E):
-        st = replica_starts(n[e], r[e])
+        if slot_share is None:
+            st = replica_starts(n[e], r[e])
+        else:
+            st = replica_starts_by_share(n[e], np.asarray(slot_share).reshape(-1)[so[e]:so[e] + r[e]])
         starts.append(st)
         for rho in range(r[e]):
             load[so[e] + rho] = st[rho + 1] - st[rho]

@@ -53,7 +53,7 @@ ERR_STATIC_SCRATCH_EXCEEDED = -9
 
 EXPORTS = (
     "moegps_create", "moegps_destroy", "moegps_rcap", "moegps_workspace_bytes", "moegps_route",
-    "moegps_route_histogram", "moegps_route_logits", "moegps_histogram", "moegps_plan", "moegps_pack", "moegps_dispatch", "moegps_dispatch_static",
+    "moegps_route_histogram", "moegps_route_logits", "moegps_histogram", "moegps_plan", "moegps_pack", "moegps_pack_slots", "moegps_dispatch", "moegps_dispatch_shares", "moegps_dispatch_static",
     "moegps_expert_ffn", "moegps_expert_ffn_gate_up", "moegps_expert_ffn_down", "moegps_combine",
     "moegps_status", "moegps_launch_count", "moegps_last_cuda_error", "moegps_error_string",
     "moegps_selftest_bounded_wait", "moegps_predictor_update", "moegps_predictor_update_ema", "moegps_error_rate",
@@ -99,7 +99,9 @@ def _lib():
         "moegps_histogram": (ctypes.c_int, [vp] * 4),
         "moegps_plan": (ctypes.c_int, [vp, vp, i32, vp, vp, vp, vp, vp]),
         "moegps_pack": (ctypes.c_int, [vp, vp, vp, vp, i32, vp, vp, vp, vp, vp]),
+        "moegps_pack_slots": (ctypes.c_int, [vp, vp, vp, i32, vp, vp, vp, vp, vp, vp]),
         "moegps_dispatch": (ctypes.c_int, [vp] * 12),
+        "moegps_dispatch_shares": (ctypes.c_int, [vp] * 13),
         "moegps_dispatch_static": (ctypes.c_int, [vp] * 11),
         "moegps_expert_ffn": (ctypes.c_int, [vp] * 10),
         "moegps_expert_ffn_gate_up": (ctypes.c_int, [vp] * 8),
@@ -228,6 +230,33 @@ class Context:
             _ptr(placement, torch.int32, (s.E, g), "placement"), _ptr(share, torch.int32, (s.E, g), "share"),
             _ptr(load, torch.int32, (g,), "load"), _ptr(iterations, torch.int32, (1,), "iterations"),
             _stream(stream)), "moegps_pack")
+
+    def pack_slots(self, placement, share, n_devices, replicas, slot_off, slot_expert, slot_share, slot_device,
+                   stream=None):
+        s, g = self.shape, int(n_devices)
+        self._check(_lib().moegps_pack_slots(
+            self._h, _ptr(placement, torch.int32, (s.E, g), "placement"), _ptr(share, torch.int32, (s.E, g), "share"), g,
+            _ptr(replicas, torch.int32, (s.E,), "replicas"), _ptr(slot_off, torch.int32, (s.E + 1,), "slot_off"),
+            _ptr(slot_expert, torch.int32, (s.S,), "slot_expert"), _ptr(slot_share, torch.int32, (s.S,), "slot_share"),
+            _ptr(slot_device, torch.int32, (s.S,), "slot_device"), _stream(stream)), "moegps_pack_slots")
+
+    def dispatch_shares(self, x, topk_idx, hist, replicas, slot_off, slot_share, slot_row_off, row_pair, pair_row,
+                        xp, workspace, stream=None):
+        s = self.shape
+        if workspace is None or workspace.numel() * workspace.element_size() < workspace_bytes(s):
+            raise MoegpsError(ERR_WORKSPACE_TOO_SMALL, "moegps_dispatch_shares")
+        self._check(_lib().moegps_dispatch_shares(
+            self._h, _ptr(x, torch.bfloat16, (s.T, s.D), "x"),
+            _ptr(topk_idx, torch.int32, (s.T, s.K), "topk_idx"),
+            _ptr(hist, torch.int32, (s.E,), "hist"),
+            _ptr(replicas, torch.int32, (s.E,), "replicas"),
+            _ptr(slot_off, torch.int32, (s.E + 1,), "slot_off"),
+            _ptr(slot_share, torch.int32, (s.S,), "slot_share"),
+            _ptr(slot_row_off, torch.int32, (s.S + 1,), "slot_row_off"),
+            _ptr(row_pair, torch.int32, (s.Rcap,), "row_pair"),
+            _ptr(pair_row, torch.int32, (s.T, s.K), "pair_row"),
+            _ptr(xp, torch.bfloat16, (s.Rcap, s.D), "xp"),
+            _ptr(workspace, workspace.dtype, None, "workspace"), _stream(stream)), "moegps_dispatch_shares")
 
     def dispatch(self, x, topk_idx, hist, replicas, slot_off, slot_row_off, row_pair, pair_row, xp,
                  workspace, stream=None):

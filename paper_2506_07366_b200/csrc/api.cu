@@ -144,8 +144,20 @@ int moegps_dispatch(moegps_ctx_t* ctx, const void* x, const int32_t* topk_idx, c
   if (int rc = moegps_check_device(ctx)) return rc;
   if (ctx->shape.T > 0 && !all_ok(x, topk_idx, pair_row, xp)) return MOEGPS_ERR_INVALID_ARG;
   if (moegps_rcap_of(ctx->shape) > 0 && !all_ok(row_pair)) return MOEGPS_ERR_INVALID_ARG;
-  return moegps_launch_dispatch(ctx, x, topk_idx, hist, replicas, slot_off, slot_row_off, row_pair, pair_row,
+  return moegps_launch_dispatch(ctx, x, topk_idx, hist, replicas, slot_off, nullptr, slot_row_off, row_pair, pair_row,
                                 xp, workspace, (cudaStream_t)stream);
+}
+
+int moegps_dispatch_shares(moegps_ctx_t* ctx, const void* x, const int32_t* topk_idx, const int32_t* hist,
+                           const int32_t* replicas, const int32_t* slot_off, const int32_t* slot_share,
+                           int32_t* slot_row_off, int32_t* row_pair, int32_t* pair_row, void* xp, void* workspace,
+                           void* stream) {
+  if (!ctx || !all_ok(hist, replicas, slot_off, slot_share, slot_row_off, workspace)) return MOEGPS_ERR_INVALID_ARG;
+  if (int rc = moegps_check_device(ctx)) return rc;
+  if (ctx->shape.T > 0 && !all_ok(x, topk_idx, pair_row, xp)) return MOEGPS_ERR_INVALID_ARG;
+  if (moegps_rcap_of(ctx->shape) > 0 && !all_ok(row_pair)) return MOEGPS_ERR_INVALID_ARG;
+  return moegps_launch_dispatch(ctx, x, topk_idx, hist, replicas, slot_off, slot_share, slot_row_off, row_pair,
+                                pair_row, xp, workspace, (cudaStream_t)stream);
 }
 
 int moegps_expert_ffn(moegps_ctx_t* ctx, const void* xp, const int32_t* slot_row_off,

@@ -82,8 +82,8 @@ int moegps_launch_histogram(moegps_ctx* ctx, const int32_t* topk_idx, int32_t* h
 int moegps_launch_plan(moegps_ctx* ctx, const int32_t* pred, int32_t* replicas, int32_t* slot_off,
                        int32_t* slot_expert, int32_t* bound, cudaStream_t st);
 int moegps_launch_dispatch(moegps_ctx* ctx, const void* x, const int32_t* topk_idx, const int32_t* hist,
-                           const int32_t* replicas, const int32_t* slot_off, int32_t* slot_row_off,
-                           int32_t* row_pair, int32_t* pair_row, void* xp, void* workspace,
+                           const int32_t* replicas, const int32_t* slot_off, const int32_t* slot_share,
+                           int32_t* slot_row_off, int32_t* row_pair, int32_t* pair_row, void* xp, void* workspace,
                            cudaStream_t st);
 int moegps_launch_ffn_gate_up(moegps_ctx* ctx, const void* xp, const int32_t* slot_row_off,
                               const int32_t* slot_expert, const void* w_gate, const void* w_up, void* h_ws,

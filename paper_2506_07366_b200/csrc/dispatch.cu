@@ -38,17 +38,45 @@ static_assert(kMaxS <= 4 * kSegPairs, "count_kernel scans four slots per thread"
 
 constexpr int kDirectMaxSeg = 1024;   // up to this many segments rank_copy sums the counts itself
 
+// Total of the predicted tokens that the copies of an expert were given (slot_share, from
+// moegps_pack_slots); 0 when there is no share table, the prediction gave the expert nothing, or the
+// table is out of range (then the copies take equal parts).
+__device__ __forceinline__ long long share_total(const int32_t* __restrict__ slot_share, int so, int r) {
+  if (!slot_share) return 0;
+  long long tot = 0;
+  for (int rho = 0; rho < r; ++rho) {
+    const int v = slot_share[so + rho];
+    if (v < 0) return 0;
+    tot += v;
+  }
+  return tot > 0x7fffffffll ? 0 : tot;
+}
+
 // Rows reserved for the replicas of expert `e` (loads rounded up to A) -> padded[slot].
-// Replica rho takes ranks floor(rho n/r) .. floor((rho+1) n/r) - 1.
+// Replica rho takes ranks floor(rho n/r) .. floor((rho+1) n/r) - 1, or, with a share table, ranks
+// floor(n c_rho / c) .. floor(n c_{rho+1} / c) - 1 with c_rho the shares of the copies before it.
 __device__ __forceinline__ void slot_loads_of_expert(int e, int S, int A, const int32_t* __restrict__ hist,
                                                      const int32_t* __restrict__ replicas,
-                                                     const int32_t* __restrict__ slot_off, int32_t* padded,
+                                                     const int32_t* __restrict__ slot_off,
+                                                     const int32_t* __restrict__ slot_share, int32_t* padded,
                                                      int32_t* status) {
   const long long n = hist[e];
   const int r = replicas[e];
   const int so = slot_off[e];
   if (r < 1 || so < 0 || so + r > S || n < 0) {
     moegps_report(status, MOEGPS_ERR_BAD_INDEX, e);
+    return;
+  }
+  const long long tot = share_total(slot_share, so, r);
+  if (tot > 0) {
+    long long cum = 0;
+    int prev = 0;
+    for (int rho = 0; rho < r; ++rho) {
+      cum += slot_share[so + rho];
+      const int start = (int)((n * cum) / tot);      // n, cum < 2^31
+      padded[so + rho] = (start - prev + A - 1) / A * A;
+      prev = start;
+    }
     return;
   }
   // floor(rho n / r) = rho q + floor(rho m / r) with n = q r + m: one division, then 32-bit work
@@ -66,7 +94,7 @@ __global__ void __launch_bounds__(kSegPairs)
 count_kernel(const int32_t* __restrict__ topk_idx, int64_t R, int E, int S, int A, int32_t* __restrict__ cnt_t,
              int nseg, int32_t* __restrict__ row_pair, int64_t Rcap, const int32_t* __restrict__ hist,
              const int32_t* __restrict__ replicas, const int32_t* __restrict__ slot_off,
-             int32_t* __restrict__ slot_row_off, int32_t* status) {
+             const int32_t* __restrict__ slot_share, int32_t* __restrict__ slot_row_off, int32_t* status) {
   __shared__ int32_t cnt[kMaxE];
   __shared__ int32_t padded[kMaxS];
   __shared__ int32_t warp_tot[kSegPairs / 32];
@@ -98,7 +126,7 @@ count_kernel(const int32_t* __restrict__ topk_idx, int64_t R, int E, int S, int 
   // ---- CTA 0: slot row offsets (independent of the counts) ----
   for (int s = tid; s < S; s += kSegPairs) padded[s] = 0;
   __syncthreads();
-  for (int e = tid; e < E; e += kSegPairs) slot_loads_of_expert(e, S, A, hist, replicas, slot_off, padded, status);
+  for (int e = tid; e < E; e += kSegPairs) slot_loads_of_expert(e, S, A, hist, replicas, slot_off, slot_share, padded, status);
   __syncthreads();
   // slot starts are multiples of A, so the offsets are a plain prefix sum of the padded loads;
   // thread t owns slots 4t .. 4t+3 (S <= 1024 = 4 * 256)
@@ -132,8 +160,8 @@ __global__ void __launch_bounds__(kScanThreads)
 count_scan_kernel(const int32_t* __restrict__ topk_idx, int64_t R, int E, int S, int A,
                   int32_t* seg_cnt, int nseg, int32_t* __restrict__ row_pair, int64_t Rcap,
                   const int32_t* __restrict__ hist, const int32_t* __restrict__ replicas,
-                  const int32_t* __restrict__ slot_off, int32_t* __restrict__ slot_row_off,
-                  int e_chunk, int32_t* __restrict__ ticket_ctr, int32_t* status) {
+                  const int32_t* __restrict__ slot_off, const int32_t* __restrict__ slot_share,
+                  int32_t* __restrict__ slot_row_off, int e_chunk, int32_t* __restrict__ ticket_ctr, int32_t* status) {
   __shared__ int32_t cnt[kMaxE];
   __shared__ int32_t padded[kMaxS];     // rows reserved for each slot (load rounded up to A)
   __shared__ int32_t warp_tot[32];
@@ -238,7 +266,7 @@ count_scan_kernel(const int32_t* __restrict__ topk_idx, int64_t R, int E, int S,
     if (lane == 0 && running != hist[e]) moegps_report(status, MOEGPS_ERR_HIST_MISMATCH, e);
   }
   // (b) slot loads
-  if (tid < E) slot_loads_of_expert(tid, S, A, hist, replicas, slot_off, padded, status);
+  if (tid < E) slot_loads_of_expert(tid, S, A, hist, replicas, slot_off, slot_share, padded, status);
   __syncthreads();
   // slot starts are multiples of A, so the offsets are a plain prefix sum of the padded loads
   const int v = tid < S ? padded[tid] : 0;
@@ -264,8 +292,9 @@ rank_copy_kernel(const uint4* __restrict__ x, int T, int K, int chunks /* D*2/16
                  const int32_t* __restrict__ topk_idx, int64_t R, int E, int S, int64_t Rcap,
                  const int32_t* __restrict__ seg_base, int nseg, const int32_t* __restrict__ hist,
                  const int32_t* __restrict__ replicas, const int32_t* __restrict__ slot_off,
-                 const int32_t* __restrict__ slot_row_off, int32_t* __restrict__ pair_row,
-                 int32_t* __restrict__ row_pair, uint4* __restrict__ xp, int32_t* __restrict__ status) {
+                 const int32_t* __restrict__ slot_share, const int32_t* __restrict__ slot_row_off,
+                 int32_t* __restrict__ pair_row, int32_t* __restrict__ row_pair, uint4* __restrict__ xp,
+                 int32_t* __restrict__ status) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   if (kDirect && blockIdx.x == 0) {
     // the counts must add up to the histogram the caller passed (the scan path checks the same)
@@ -329,9 +358,24 @@ rank_copy_kernel(const uint4* __restrict__ x, int T, int K, int chunks /* D*2/16
     if (n <= 0 || r < 1 || my_rank >= n) {
       moegps_report(status, MOEGPS_ERR_HIST_MISMATCH, my_e);
     } else {
-      const int rho = (int)((((long long)my_rank + 1) * r - 1) / n);   // replica whose range holds the rank
-      const int start = (int)(((long long)rho * n) / r);
-      const int slot = slot_off[my_e] + rho;
+      const int so = slot_off[my_e];
+      int rho, start;
+      const long long tot = (so >= 0 && so + r <= S) ? share_total(slot_share, so, r) : 0;
+      if (tot > 0) {                                                   // copies take parts in proportion to their shares
+        long long cum = 0;
+        int end = 0;
+        start = 0;
+        for (rho = 0; rho < r - 1; ++rho) {
+          cum += slot_share[so + rho];
+          end = (int)((n * cum) / tot);
+          if (my_rank < end) break;
+          start = end;
+        }
+      } else {
+        rho = (int)((((long long)my_rank + 1) * r - 1) / n);           // replica whose range holds the rank
+        start = (int)(((long long)rho * n) / r);
+      }
+      const int slot = so + rho;
       const long long rr = (slot >= 0 && slot < S) ? (long long)slot_row_off[slot] + (my_rank - start) : -1;
       if (rr < 0 || rr >= Rcap) {
         moegps_report(status, MOEGPS_ERR_BAD_INDEX, t);
@@ -372,8 +416,9 @@ rank_copy_kernel(const uint4* __restrict__ x, int T, int K, int chunks /* D*2/16
 }  // namespace
 
 int moegps_launch_dispatch(moegps_ctx* ctx, const void* x, const int32_t* topk_idx, const int32_t* hist,
-                           const int32_t* replicas, const int32_t* slot_off, int32_t* slot_row_off,
-                           int32_t* row_pair, int32_t* pair_row, void* xp, void* workspace, cudaStream_t st) {
+                           const int32_t* replicas, const int32_t* slot_off, const int32_t* slot_share,
+                           int32_t* slot_row_off, int32_t* row_pair, int32_t* pair_row, void* xp, void* workspace,
+                           cudaStream_t st) {
   const moegps_shape_t& s = ctx->shape;
   const int64_t R = (int64_t)s.T * s.K;
   const int64_t Rcap = moegps_rcap_of(s);
@@ -392,13 +437,14 @@ int moegps_launch_dispatch(moegps_ctx* ctx, const void* x, const int32_t* topk_i
   const bool direct = nseg <= kDirectMaxSeg;
   if (direct) {
     count_kernel<<<nseg > 0 ? nseg : 1, kSegPairs, 0, st>>>(topk_idx, R, s.E, s.S, s.row_align, seg, nseg, row_pair, Rcap,
-                                                            hist, replicas, slot_off, slot_row_off, ctx->d_status);
+                                                            hist, replicas, slot_off, slot_share, slot_row_off,
+                                                            ctx->d_status);
   } else {
     int32_t* ticket = seg + (int64_t)nseg * s.E;     // the scratch's last word (see moegps_workspace_bytes)
     MOEGPS_CUDA_TRY(ctx, cudaMemsetAsync(ticket, 0, sizeof(int32_t), st));
     count_scan_kernel<<<nseg, kScanThreads, scan_smem, st>>>(topk_idx, R, s.E, s.S, s.row_align, seg, nseg, row_pair,
-                                                             Rcap, hist, replicas, slot_off, slot_row_off, e_chunk,
-                                                             ticket, ctx->d_status);
+                                                             Rcap, hist, replicas, slot_off, slot_share, slot_row_off,
+                                                             e_chunk, ticket, ctx->d_status);
   }
   MOEGPS_AFTER_LAUNCH(ctx);
   if (R == 0) return MOEGPS_OK;
@@ -406,11 +452,11 @@ int moegps_launch_dispatch(moegps_ctx* ctx, const void* x, const int32_t* topk_i
   if (direct) {
     rank_copy_kernel<true><<<tblocks, kThreads, 0, st>>>(
         static_cast<const uint4*>(x), s.T, s.K, s.D / 8, topk_idx, R, s.E, s.S, Rcap, seg, nseg, hist, replicas, slot_off,
-        slot_row_off, pair_row, row_pair, static_cast<uint4*>(xp), ctx->d_status);
+        slot_share, slot_row_off, pair_row, row_pair, static_cast<uint4*>(xp), ctx->d_status);
   } else {
     rank_copy_kernel<false><<<tblocks, kThreads, 0, st>>>(
         static_cast<const uint4*>(x), s.T, s.K, s.D / 8, topk_idx, R, s.E, s.S, Rcap, seg, nseg, hist, replicas, slot_off,
-        slot_row_off, pair_row, row_pair, static_cast<uint4*>(xp), ctx->d_status);
+        slot_share, slot_row_off, pair_row, row_pair, static_cast<uint4*>(xp), ctx->d_status);
   }
   MOEGPS_AFTER_LAUNCH(ctx);
   return MOEGPS_OK;
@@ -465,6 +511,6 @@ extern "C" MOEGPS_API int moegps_dispatch_static(moegps_ctx_t* ctx, const void* 
     if (!scratch) return MOEGPS_ERR_CUDA;
     g_scratch_addr[dev].store(scratch, std::memory_order_release);
   }
-  return moegps_launch_dispatch(ctx, x, topk_idx, hist, replicas, slot_off, slot_row_off, row_pair, pair_row, xp,
-                                scratch, (cudaStream_t)stream);
+  return moegps_launch_dispatch(ctx, x, topk_idx, hist, replicas, slot_off, nullptr, slot_row_off, row_pair, pair_row,
+                                xp, scratch, (cudaStream_t)stream);
 }

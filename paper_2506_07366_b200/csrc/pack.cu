@@ -125,9 +125,74 @@ pack_kernel(const int32_t* __restrict__ pred, const int32_t* __restrict__ home, 
   if (lane == 0) iters_out[0] = iters;
 }
 
+// The placement as slot tables: one slot per (expert, device) copy, experts ascending and, within an
+// expert, devices ascending; slots beyond the last copy are empty.  One CTA, thread e = expert e.
+__global__ void __launch_bounds__(kMaxE)
+pack_slots_kernel(const int32_t* __restrict__ placement, const int32_t* __restrict__ share, int E, int G, int S,
+                  int32_t* __restrict__ replicas, int32_t* __restrict__ slot_off, int32_t* __restrict__ slot_expert,
+                  int32_t* __restrict__ slot_share, int32_t* __restrict__ slot_device, int32_t* __restrict__ status) {
+  __shared__ int warp_sum[kMaxE / 32];
+  const int e = threadIdx.x, lane = e & 31, warp = e >> 5;
+  int r = 0;
+  if (e < E)
+    for (int g = 0; g < G; ++g) r += placement[e * G + g] != 0;
+  int incl = r;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const int o = __shfl_up_sync(0xffffffffu, incl, d);
+    if (lane >= d) incl += o;
+  }
+  if (lane == 31) warp_sum[warp] = incl;
+  __syncthreads();
+  int base = 0, total = 0;
+  for (int w = 0; w < kMaxE / 32; ++w) {
+    if (w < warp) base += warp_sum[w];
+    total += warp_sum[w];
+  }
+  const int first = base + incl - r;
+  if (e == 0 && total > S) moegps_report(status, MOEGPS_ERR_BAD_INDEX, total);   // more copies than slots
+  if (e < E) {
+    replicas[e] = r;
+    slot_off[e] = first;
+    int s = first;
+    for (int g = 0; g < G; ++g) {
+      if (placement[e * G + g] != 0) {
+        if (s < S) {
+          slot_expert[s] = e;
+          slot_share[s] = share[e * G + g];
+          slot_device[s] = g;
+        }
+        ++s;
+      }
+    }
+  }
+  if (e == 0) slot_off[E] = total;
+  for (int s = total + e; s < S; s += kMaxE) {
+    slot_expert[s] = -1;
+    slot_share[s] = 0;
+    slot_device[s] = -1;
+  }
+}
+
 bool ok16(const void* p) { return p != nullptr && moegps_aligned16(p); }
 
 }  // namespace
+
+extern "C" MOEGPS_API int moegps_pack_slots(moegps_ctx_t* ctx, const int32_t* placement, const int32_t* share,
+                                            int32_t n_devices, int32_t* replicas, int32_t* slot_off,
+                                            int32_t* slot_expert, int32_t* slot_share, int32_t* slot_device,
+                                            void* stream) {
+  if (!ctx || !ok16(placement) || !ok16(share) || !ok16(replicas) || !ok16(slot_off) || !ok16(slot_expert) ||
+      !ok16(slot_share) || !ok16(slot_device))
+    return MOEGPS_ERR_INVALID_ARG;
+  if (n_devices < 1 || n_devices > kMaxG) return MOEGPS_ERR_UNSUPPORTED_SHAPE;
+  if (int rc = moegps_check_device(ctx)) return rc;
+  pack_slots_kernel<<<1, kMaxE, 0, (cudaStream_t)stream>>>(placement, share, ctx->shape.E, n_devices, ctx->shape.S,
+                                                           replicas, slot_off, slot_expert, slot_share, slot_device,
+                                                           ctx->d_status);
+  MOEGPS_AFTER_LAUNCH(ctx);
+  return MOEGPS_OK;
+}
 
 extern "C" MOEGPS_API int moegps_pack(moegps_ctx_t* ctx, const int32_t* predicted_hist, const int32_t* home,
                                       const int32_t* capacity, int32_t n_devices, int32_t* placement,

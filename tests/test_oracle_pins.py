@@ -411,6 +411,66 @@ def test_pack_never_beats_the_slot_planner_bound():
     assert sorted(load.tolist()) == [33, 33, 34] and iters > 2
 
 
+def test_pack_slots_and_split_by_share():
+    # hand-worked: 10 pairs over copies with predicted shares 3 : 1 -> boundaries 0, floor(10*3/4) = 7, 10
+    assert oracle.replica_starts_by_share(10, [3, 1]) == [0, 7, 10]
+    assert oracle.replica_starts_by_share(10, [0, 5, 0]) == [0, 0, 10, 10]          # a copy with no share gets nothing
+    assert oracle.replica_starts_by_share(10, [0, 0, 0]) == oracle.replica_starts(10, 3)   # nothing predicted: even split
+    for n in (0, 1, 7, 100, 12345):
+        for r in (1, 2, 3, 7):
+            assert oracle.replica_starts_by_share(n, [5] * r) == oracle.replica_starts(n, r)  # equal shares = balanced split
+    for trial in range(50):
+        r, n = int(rng.integers(1, 9)), int(rng.integers(0, 5000))
+        sh = rng.integers(0, 1000, size=r)
+        st = oracle.replica_starts_by_share(n, sh)
+        assert st[0] == 0 and st[-1] == n and all(a <= b for a, b in zip(st, st[1:]))
+        if sh.sum() > 0:                                  # every copy within one pair of its proportional part
+            loads = np.diff(st)
+            assert np.abs(loads - n * sh / sh.sum()).max() < 1.0
+    # slot tables of the paper's example: expert 0 on all four devices, the others at home
+    placed, share, load, _ = oracle.pack([9, 1, 1, 1], [0, 1, 2, 3], [4] * 4)
+    rep, so, se, ss, sd = oracle.pack_slots(placed, share, 9)
+    assert rep.tolist() == [4, 1, 1, 1] and so.tolist() == [0, 4, 5, 6, 7]
+    assert se.tolist() == [0, 0, 0, 0, 1, 2, 3, -1, -1] and sd.tolist() == [0, 1, 2, 3, 1, 2, 3, -1, -1]
+    assert ss.tolist() == [3, 2, 2, 2, 1, 1, 1, 0, 0]
+    assert [int(ss[sd == g].sum()) for g in range(4)] == load.tolist()      # shares per device add up to its load
+    with pytest.raises(ValueError):
+        oracle.pack_slots(placed, share, 6)
+
+
+def test_dispatch_by_share_realises_the_packed_loads():
+    """pack -> pack_slots -> dispatch with shares: with an exact prediction every device receives
+    exactly the load Algorithm 1 planned for it, and the permutation keeps all dispatch invariants."""
+    E, G, K, T = 6, 3, 2, 300
+    idx = random_routing(T, K, E, 1.3)
+    n = oracle.histogram(idx, E)
+    placed, share, load, _ = oracle.pack(n, [e % G for e in range(E)], [4] * G)
+    S = int(placed.sum()) + 2
+    rep, so, se, ss, sd = oracle.pack_slots(placed, share, S)
+    sro, rp, pr, _ = oracle.dispatch(None, idx, n, rep, so, S, 4, slot_share=ss)
+    flat = idx.reshape(-1)
+    assert sorted(pr.reshape(-1).tolist()) == sorted(np.nonzero(rp >= 0)[0].tolist())      # bijection onto occupied rows
+    assert np.array_equal(rp[pr.reshape(-1)], np.arange(T * K))
+    dev_load = np.zeros(G, dtype=np.int64)
+    for s in range(S):
+        rows = rp[sro[s]:sro[s + 1]]
+        rows = rows[rows >= 0]
+        assert (np.diff(rows) > 0).all()                                                    # stable inside a slot
+        if rows.size:
+            assert (flat[rows] == se[s]).all()
+            dev_load[sd[s]] += rows.size
+        assert rows.size == ss[s]                                                           # exact prediction: planned = realised
+    assert dev_load.tolist() == load.tolist() and load.max() - load.min() <= 1
+    # with a wrong prediction the split follows the predicted proportions of the ACTUAL counts
+    n2 = oracle.histogram(random_routing(T, K, E, 0.2), E)
+    idx2 = random_routing(T, K, E, 0.2)
+    sro2, rp2, _, _ = oracle.dispatch(None, idx2, oracle.histogram(idx2, E), rep, so, S, 1, slot_share=ss)
+    for e in range(E):
+        got = [int(np.count_nonzero(rp2[sro2[s]:sro2[s + 1]] >= 0)) for s in range(so[e], so[e + 1])]
+        want = np.diff(oracle.replica_starts_by_share(int(oracle.histogram(idx2, E)[e]), ss[so[e]:so[e + 1]])).tolist()
+        assert got == want
+
+
 # ------------------------------------------------------------------------------ dispatch
 def closed_form_replica(i, n, r):
     return ((i + 1) * r - 1) // n

@@ -43,12 +43,15 @@ def run_both(ctx, shape, x, idx, pred):
         pr = torch.full((shape.T, shape.K), -5, **i32)
         xp = torch.full((shape.Rcap, shape.D), 0x3C3C, dtype=torch.int16, device=DEV).view(torch.bfloat16)
         if static:
-            # the claim "allocates nothing": neither the driver's nor torch's view of device memory moves
+            # the claim "allocates nothing": the driver's free memory does not shrink and torch's
+            # allocator sees no new request while the call runs (frees by the garbage collector may happen)
             torch.cuda.synchronize()
-            free0, alloc0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
+            free0 = torch.cuda.mem_get_info()[0]
+            requests0 = torch.cuda.memory_stats()["allocation.all.allocated"]
             ctx.dispatch_static(x, idx, hist, rep, so, sro, rp, pr, xp)
             torch.cuda.synchronize()
-            assert torch.cuda.mem_get_info()[0] == free0 and torch.cuda.memory_allocated() == alloc0
+            assert torch.cuda.mem_get_info()[0] >= free0
+            assert torch.cuda.memory_stats()["allocation.all.allocated"] == requests0
         else:
             ws = torch.empty(binding.workspace_bytes(shape), dtype=torch.uint8, device=DEV)
             ctx.dispatch(x, idx, hist, rep, so, sro, rp, pr, xp, ws)
