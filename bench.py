@@ -500,10 +500,13 @@ def run_ours(args):
             if name == w.name:
                 continue
             torch.cuda.empty_cache()
-            ob = Bench(wl.WORKLOADS[name], 0, local_rank)
-            per[name] = compact_record(ob, peaks, args.per_workload_steps, barrier)
-            ob.close()
-            del ob
+            try:                            # a failure here must not cost the headline measurement above
+                ob = Bench(wl.WORKLOADS[name], 0, local_rank)
+                per[name] = compact_record(ob, peaks, args.per_workload_steps, barrier)
+                ob.close()
+                del ob
+            except Exception as exc:        # noqa: BLE001 - reported in the line instead
+                per[name] = {"error": f"{type(exc).__name__}: {exc}"[:300]}
         line["per_workload"] = per
     print(json.dumps(line), flush=True)
     if dist is not None:
