@@ -236,9 +236,11 @@ class Bench:
     def step(self, record: bool):
         L, c, w = self.layer, self.ctx, self.w
         c.plan(self.pred_dev, w.S, L.replicas, L.slot_off, L.slot_expert, L.bound)
-        c.route_histogram(self.x, self.wr, self.bias, L.topk_idx, L.topk_w, L.hist)     # route + histogram fused
-        c.dispatch(self.x, L.topk_idx, L.hist, L.replicas, L.slot_off, L.slot_row_off, L.row_pair, L.pair_row,
-                   L.xp, L.workspace)
+        # route + histogram + what dispatch needs (counts, slot row offsets) in one kernel, dispatch in one
+        c.route_prepare(self.x, self.wr, self.bias, L.replicas, L.slot_off, L.topk_idx, L.topk_w, L.hist,
+                        L.slot_row_off, L.workspace)
+        c.dispatch_prepared(self.x, L.topk_idx, L.hist, L.replicas, L.slot_off, L.slot_row_off, L.row_pair,
+                            L.pair_row, L.xp, L.workspace)
         stream = torch.cuda.current_stream()
         if record:
             a, b, e = (torch.cuda.Event(enable_timing=True) for _ in range(3))
@@ -341,6 +343,13 @@ class Bench:
             ("dispatch", lambda: c.dispatch(self.x, L.topk_idx, L.hist, L.replicas, L.slot_off, L.slot_row_off,
                                             L.row_pair, L.pair_row, L.xp, L.workspace),
              2.0 * T * D + 2.0 * R * D + 12.0 * R, None),
+            ("route_prepare", lambda: c.route_prepare(self.x, self.wr, self.bias, L.replicas, L.slot_off, L.topk_idx,
+                                                      L.topk_w, L.hist, L.slot_row_off, L.workspace),
+             2.0 * T * D + 2.0 * E * D + 8.0 * T * K, 2.0 * T * D * E),
+            ("dispatch_prepared", lambda: c.dispatch_prepared(self.x, L.topk_idx, L.hist, L.replicas, L.slot_off,
+                                                              L.slot_row_off, L.row_pair, L.pair_row, L.xp,
+                                                              L.workspace),
+             2.0 * T * D + 2.0 * R * D + 12.0 * R, None),
             ("expert_ffn_gate_up", lambda: c.expert_ffn_gate_up(L.xp, L.slot_row_off, L.slot_expert, self.w1, self.w3,
                                                                 L.h_ws), None, 4.0 * R * D * F),
             ("expert_ffn_down", lambda: c.expert_ffn_down(L.h_ws, L.slot_row_off, L.slot_expert, self.w2, L.yp),
@@ -407,9 +416,10 @@ def compact_record(b: Bench, peaks, steps: int, barrier) -> dict:
             "down_frac_of_burst_peak": ffn["down_frac_of_burst_peak"],
             "gate_up_frac_of_hbm_peak": ffn["gate_up_frac_of_hbm_peak"],
             "down_frac_of_hbm_peak": ffn["down_frac_of_hbm_peak"],
-            "cold_l2_us": {k: round(calls[k]["us"], 2) for k in ("route_histogram", "dispatch", "combine", "plan")},
+            "cold_l2_us": {k: round(calls[k]["us"], 2)
+                           for k in ("route_prepare", "dispatch_prepared", "combine", "plan")},
             "frac_of_hbm_peak": {k: round(calls[k]["frac_of_hbm_peak"], 3)
-                                 for k in ("route_histogram", "dispatch", "combine")},
+                                 for k in ("route_prepare", "dispatch_prepared", "combine")},
             "skewness": stats["skewness"], "skewness_after_plan": stats["skewness_after_plan"]}
 
 

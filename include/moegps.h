@@ -76,8 +76,9 @@ typedef struct moegps_shape {
 
 typedef struct moegps_ctx moegps_ctx_t;   /* opaque: shape, device id, device status word, cached TMA descriptors */
 
-/* Create / destroy a context on CUDA device `device`.  Allocates the (16-byte) device status word;
- * this is the only device allocation the library ever makes. */
+/* Create / destroy a context on CUDA device `device`.  Allocates one small block of device memory
+ * (about 1 KiB: the status word and the router's histogram accumulators); this is the only device
+ * allocation the library ever makes. */
 MOEGPS_API int moegps_create(moegps_ctx_t** out, const moegps_shape_t* shape, int device);
 MOEGPS_API int moegps_destroy(moegps_ctx_t* ctx);
 
@@ -100,10 +101,34 @@ MOEGPS_API int moegps_route(moegps_ctx_t* ctx, const void* x, const void* w_rout
 /* route_histogram - moegps_route and moegps_histogram in one kernel: the router's epilogue also
  * counts the selections per expert (the n_e of the paper's Eq. 1 with N = T*K), so the indices are
  * not read back from memory and one launch is saved.  Same arguments and results as moegps_route,
- * plus hist: int32 [E], fully overwritten (zeroed on the stream, then accumulated with integer
- * atomics: exact and deterministic).  Bit-identical to moegps_route followed by moegps_histogram. */
+ * plus hist: int32 [E], fully overwritten.  The counts are summed with integer atomics (exact and
+ * deterministic) in accumulators that belong to the context; the CTA that finishes last copies them
+ * to hist and leaves the accumulators at zero.  Two such calls of ONE context must therefore not
+ * overlap on the GPU (issue them on one stream, or order them with events); different contexts are
+ * independent.  Bit-identical to moegps_route followed by moegps_histogram. */
 MOEGPS_API int moegps_route_histogram(moegps_ctx_t* ctx, const void* x, const void* w_router, const float* bias,
                                       int32_t* topk_idx, float* topk_w, int32_t* hist, void* stream);
+
+/* route_prepare + dispatch_prepared - the same results as moegps_route_histogram followed by
+ * moegps_dispatch, in two launches instead of four.  The router's epilogue already holds, per CTA,
+ * the per-expert counts of the token rows that CTA owns; route_prepare stores them as the columns of
+ * the count matrix that dispatch ranks pairs with (into `workspace`), and the CTA that finishes last
+ * derives slot_row_off from the finished histogram and the plan; dispatch_prepared then only ranks,
+ * places and copies (and marks padding rows of row_pair with -1).  Copies of an expert share its
+ * pairs evenly (as in moegps_dispatch).  Bit-identical to the separate calls.
+ * route_prepare: x, w_router, bias, topk_idx, topk_w, hist as in moegps_route_histogram; replicas,
+ * slot_off from moegps_plan; slot_row_off: int32 [S+1] (output); workspace:
+ * moegps_workspace_bytes(shape) bytes, written here and read by dispatch_prepared (the layout is
+ * private to the library: pass the same buffer, untouched, on the same stream).
+ * dispatch_prepared: arguments as moegps_dispatch, except that slot_row_off and workspace are inputs. */
+MOEGPS_API int moegps_route_prepare(moegps_ctx_t* ctx, const void* x, const void* w_router, const float* bias,
+                                    const int32_t* replicas, const int32_t* slot_off, int32_t* topk_idx,
+                                    float* topk_w, int32_t* hist, int32_t* slot_row_off, void* workspace,
+                                    void* stream);
+MOEGPS_API int moegps_dispatch_prepared(moegps_ctx_t* ctx, const void* x, const int32_t* topk_idx,
+                                        const int32_t* hist, const int32_t* replicas, const int32_t* slot_off,
+                                        const int32_t* slot_row_off, int32_t* row_pair, int32_t* pair_row,
+                                        void* xp, const void* workspace, void* stream);
 
 /* Debug companion of moegps_route: also stores the fp32 logits (fp32 [T,E]) the selection was made on. */
 MOEGPS_API int moegps_route_logits(moegps_ctx_t* ctx, const void* x, const void* w_router, const float* bias,
@@ -140,8 +165,9 @@ MOEGPS_API int moegps_plan(moegps_ctx_t* ctx, const int32_t* predicted_hist, int
  * there); n_devices = G in [1,64].
  * placement: int32 [E,G] of 0/1; share: int32 [E,G]; load: int32 [G] (column sums of share);
  * iterations: int32 [1] (moves made).  All device pointers, 16-byte aligned (iterations: 4).
- * A home outside [0,G), a negative count or an over-full initial placement is reported as
- * MOEGPS_ERR_BAD_INDEX and the outputs then describe the (clamped) initial placement.
+ * A home outside [0,G), a negative count, counts that add up to more than 2^31-1 or an over-full
+ * initial placement is reported as MOEGPS_ERR_BAD_INDEX and the outputs then describe the (clamped)
+ * initial placement.
  * This call plans only: mapping its placement onto devices and the all-to-all between them are not
  * part of this single-device library. */
 MOEGPS_API int moegps_pack(moegps_ctx_t* ctx, const int32_t* predicted_hist, const int32_t* home,

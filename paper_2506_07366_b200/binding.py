@@ -53,7 +53,7 @@ ERR_STATIC_SCRATCH_EXCEEDED = -9
 
 EXPORTS = (
     "moegps_create", "moegps_destroy", "moegps_rcap", "moegps_workspace_bytes", "moegps_route",
-    "moegps_route_histogram", "moegps_route_logits", "moegps_histogram", "moegps_plan", "moegps_pack", "moegps_pack_slots", "moegps_dispatch", "moegps_dispatch_shares", "moegps_dispatch_static",
+    "moegps_route_histogram", "moegps_route_prepare", "moegps_dispatch_prepared", "moegps_route_logits", "moegps_histogram", "moegps_plan", "moegps_pack", "moegps_pack_slots", "moegps_dispatch", "moegps_dispatch_shares", "moegps_dispatch_static",
     "moegps_expert_ffn", "moegps_expert_ffn_gate_up", "moegps_expert_ffn_down", "moegps_combine",
     "moegps_status", "moegps_launch_count", "moegps_last_cuda_error", "moegps_error_string",
     "moegps_selftest_bounded_wait", "moegps_predictor_update", "moegps_predictor_update_ema", "moegps_error_rate",
@@ -95,6 +95,8 @@ def _lib():
         "moegps_workspace_bytes": (ctypes.c_size_t, [ctypes.POINTER(moegps_shape_t)]),
         "moegps_route": (ctypes.c_int, [vp] * 7),
         "moegps_route_histogram": (ctypes.c_int, [vp] * 8),
+        "moegps_route_prepare": (ctypes.c_int, [vp] * 12),
+        "moegps_dispatch_prepared": (ctypes.c_int, [vp] * 12),
         "moegps_route_logits": (ctypes.c_int, [vp] * 6),
         "moegps_histogram": (ctypes.c_int, [vp] * 4),
         "moegps_plan": (ctypes.c_int, [vp, vp, i32, vp, vp, vp, vp, vp]),
@@ -198,6 +200,40 @@ class Context:
             _ptr(topk_idx, torch.int32, (s.T, s.K), "topk_idx"),
             _ptr(topk_w, torch.float32, (s.T, s.K), "topk_w"),
             _ptr(hist, torch.int32, (s.E,), "hist"), _stream(stream)), "moegps_route_histogram")
+
+    def route_prepare(self, x, w_router, bias, replicas, slot_off, topk_idx, topk_w, hist, slot_row_off, workspace,
+                      stream=None):
+        s = self.shape
+        if workspace is None or workspace.numel() * workspace.element_size() < workspace_bytes(s):
+            raise MoegpsError(ERR_WORKSPACE_TOO_SMALL, "moegps_route_prepare")
+        self._check(_lib().moegps_route_prepare(
+            self._h, _ptr(x, torch.bfloat16, (s.T, s.D), "x"),
+            _ptr(w_router, torch.bfloat16, (s.E, s.D), "w_router"),
+            _ptr(bias, torch.float32, (s.E,), "bias", allow_none=True),
+            _ptr(replicas, torch.int32, (s.E,), "replicas"),
+            _ptr(slot_off, torch.int32, (s.E + 1,), "slot_off"),
+            _ptr(topk_idx, torch.int32, (s.T, s.K), "topk_idx"),
+            _ptr(topk_w, torch.float32, (s.T, s.K), "topk_w"),
+            _ptr(hist, torch.int32, (s.E,), "hist"),
+            _ptr(slot_row_off, torch.int32, (s.S + 1,), "slot_row_off"),
+            _ptr(workspace, workspace.dtype, None, "workspace"), _stream(stream)), "moegps_route_prepare")
+
+    def dispatch_prepared(self, x, topk_idx, hist, replicas, slot_off, slot_row_off, row_pair, pair_row, xp,
+                          workspace, stream=None):
+        s = self.shape
+        if workspace is None or workspace.numel() * workspace.element_size() < workspace_bytes(s):
+            raise MoegpsError(ERR_WORKSPACE_TOO_SMALL, "moegps_dispatch_prepared")
+        self._check(_lib().moegps_dispatch_prepared(
+            self._h, _ptr(x, torch.bfloat16, (s.T, s.D), "x"),
+            _ptr(topk_idx, torch.int32, (s.T, s.K), "topk_idx"),
+            _ptr(hist, torch.int32, (s.E,), "hist"),
+            _ptr(replicas, torch.int32, (s.E,), "replicas"),
+            _ptr(slot_off, torch.int32, (s.E + 1,), "slot_off"),
+            _ptr(slot_row_off, torch.int32, (s.S + 1,), "slot_row_off"),
+            _ptr(row_pair, torch.int32, (s.Rcap,), "row_pair"),
+            _ptr(pair_row, torch.int32, (s.T, s.K), "pair_row"),
+            _ptr(xp, torch.bfloat16, (s.Rcap, s.D), "xp"),
+            _ptr(workspace, workspace.dtype, None, "workspace"), _stream(stream)), "moegps_dispatch_prepared")
 
     def route_logits(self, x, w_router, bias, logits, stream=None):
         s = self.shape

@@ -12,7 +12,7 @@ CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libmoegps.so")
 SOURCES = ["api.cu", "route.cu", "histogram.cu", "plan.cu", "pack.cu", "dispatch.cu", "expert_ffn.cu", "combine.cu",
            "predictor.cu", "selftest.cu"]
-HEADERS = ["common.cuh", "sm100.cuh", "route_epilogue.cuh"]
+HEADERS = ["common.cuh", "sm100.cuh", "route_epilogue.cuh", "slot_offsets.cuh"]
 
 
 def _nvcc() -> str:

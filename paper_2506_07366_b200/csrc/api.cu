@@ -52,12 +52,15 @@ int moegps_create(moegps_ctx_t** out, const moegps_shape_t* shape, int device) {
   ctx->dispatch_attr_done = false;
   ctx->pack_attr_done = false;
   ctx->d_status = nullptr;
+  ctx->d_route_acc = nullptr;
   int prev = 0;
   cudaGetDevice(&prev);
   cudaError_t e = cudaSetDevice(device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
-  if (e == cudaSuccess) e = cudaMalloc(&ctx->d_status, 4 * sizeof(int32_t));
-  if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, 4 * sizeof(int32_t));
+  constexpr size_t kCtxWords = 4 + 256 + 4;      // status word, router accumulators, router ticket
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->d_status, kCtxWords * sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, kCtxWords * sizeof(int32_t));
+  ctx->d_route_acc = ctx->d_status ? ctx->d_status + 4 : nullptr;
   cudaSetDevice(prev);
   if (e != cudaSuccess) {
     if (ctx->d_status) cudaFree(ctx->d_status);
@@ -84,8 +87,13 @@ size_t moegps_workspace_bytes(const moegps_shape_t* shape) {
   if (check_shape(shape) != MOEGPS_OK) return 0;
   const int64_t R = (int64_t)shape->T * shape->K;
   const int64_t nseg = (R + kSegPairs - 1) / kSegPairs;
-  // the per-(segment, expert) count matrix + one word for the scan path's ticket counter
-  size_t bytes = ((size_t)(nseg > 0 ? nseg : 1) * shape->E + 1) * sizeof(int32_t);
+  // the per-(segment, expert) count matrix + one word for the scan path's ticket counter; or, for
+  // the fused form (moegps_route_prepare), one column per router CTA: the router runs one CTA per
+  // 128-token tile, or splits the tiles over up to 8 CTAs while the grid stays within about 1.25x
+  // the SM count (bounded here by 320 CTAs)
+  const int64_t tiles = ((int64_t)shape->T + 127) / 128;
+  const int64_t cols = nseg > (tiles > 320 ? tiles : 320) ? nseg : (tiles > 320 ? tiles : 320);
+  size_t bytes = ((size_t)cols * shape->E + 1) * sizeof(int32_t);
   return (bytes + 255) & ~(size_t)255;
 }
 
@@ -96,7 +104,7 @@ int moegps_route(moegps_ctx_t* ctx, const void* x, const void* w_router, const f
   if (ctx->shape.T == 0) return MOEGPS_OK;          // nothing to route (empty tensors have no address)
   if (!all_ok(x, w_router, topk_idx, topk_w)) return MOEGPS_ERR_INVALID_ARG;
   if (bias && (reinterpret_cast<uintptr_t>(bias) & 3u)) return MOEGPS_ERR_INVALID_ARG;
-  return moegps_launch_route(ctx, x, w_router, bias, topk_idx, topk_w, nullptr, nullptr, (cudaStream_t)stream);
+  return moegps_launch_route(ctx, x, w_router, bias, topk_idx, topk_w, nullptr, nullptr, nullptr, (cudaStream_t)stream);
 }
 
 int moegps_route_histogram(moegps_ctx_t* ctx, const void* x, const void* w_router, const float* bias,
@@ -108,7 +116,35 @@ int moegps_route_histogram(moegps_ctx_t* ctx, const void* x, const void* w_route
                ? MOEGPS_OK : MOEGPS_ERR_CUDA;
   if (!all_ok(x, w_router, topk_idx, topk_w)) return MOEGPS_ERR_INVALID_ARG;
   if (bias && (reinterpret_cast<uintptr_t>(bias) & 3u)) return MOEGPS_ERR_INVALID_ARG;
-  return moegps_launch_route(ctx, x, w_router, bias, topk_idx, topk_w, nullptr, hist, (cudaStream_t)stream);
+  return moegps_launch_route(ctx, x, w_router, bias, topk_idx, topk_w, nullptr, hist, nullptr, (cudaStream_t)stream);
+}
+
+int moegps_route_prepare(moegps_ctx_t* ctx, const void* x, const void* w_router, const float* bias,
+                         const int32_t* replicas, const int32_t* slot_off, int32_t* topk_idx, float* topk_w,
+                         int32_t* hist, int32_t* slot_row_off, void* workspace, void* stream) {
+  if (!ctx || !all_ok(replicas, slot_off, hist, slot_row_off, workspace)) return MOEGPS_ERR_INVALID_ARG;
+  if (int rc = moegps_check_device(ctx)) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (ctx->shape.T == 0) {                          // no tokens: empty histogram, every slot empty
+    MOEGPS_CUDA_TRY(ctx, cudaMemsetAsync(hist, 0, sizeof(int32_t) * ctx->shape.E, st));
+    MOEGPS_CUDA_TRY(ctx, cudaMemsetAsync(slot_row_off, 0, sizeof(int32_t) * (ctx->shape.S + 1), st));
+    return MOEGPS_OK;
+  }
+  if (!all_ok(x, w_router, topk_idx, topk_w)) return MOEGPS_ERR_INVALID_ARG;
+  if (bias && (reinterpret_cast<uintptr_t>(bias) & 3u)) return MOEGPS_ERR_INVALID_ARG;
+  const moegps_route_fused fused = {static_cast<int32_t*>(workspace), replicas, slot_off, slot_row_off};
+  return moegps_launch_route(ctx, x, w_router, bias, topk_idx, topk_w, nullptr, hist, &fused, st);
+}
+
+int moegps_dispatch_prepared(moegps_ctx_t* ctx, const void* x, const int32_t* topk_idx, const int32_t* hist,
+                             const int32_t* replicas, const int32_t* slot_off, const int32_t* slot_row_off,
+                             int32_t* row_pair, int32_t* pair_row, void* xp, const void* workspace, void* stream) {
+  if (!ctx || !all_ok(hist, replicas, slot_off, slot_row_off, workspace)) return MOEGPS_ERR_INVALID_ARG;
+  if (int rc = moegps_check_device(ctx)) return rc;
+  if (ctx->shape.T == 0) return MOEGPS_OK;          // nothing routed: no row is occupied, no padding exists
+  if (!all_ok(x, topk_idx, pair_row, xp, row_pair)) return MOEGPS_ERR_INVALID_ARG;
+  return moegps_launch_dispatch_prepared(ctx, x, topk_idx, hist, replicas, slot_off, slot_row_off, row_pair, pair_row,
+                                         xp, workspace, (cudaStream_t)stream);
 }
 
 int moegps_route_logits(moegps_ctx_t* ctx, const void* x, const void* w_router, const float* bias,
@@ -118,7 +154,7 @@ int moegps_route_logits(moegps_ctx_t* ctx, const void* x, const void* w_router, 
   if (ctx->shape.T == 0) return MOEGPS_OK;
   if (!all_ok(x, w_router, logits)) return MOEGPS_ERR_INVALID_ARG;
   if (bias && (reinterpret_cast<uintptr_t>(bias) & 3u)) return MOEGPS_ERR_INVALID_ARG;
-  return moegps_launch_route(ctx, x, w_router, bias, nullptr, nullptr, logits, nullptr, (cudaStream_t)stream);
+  return moegps_launch_route(ctx, x, w_router, bias, nullptr, nullptr, logits, nullptr, nullptr, (cudaStream_t)stream);
 }
 
 int moegps_histogram(moegps_ctx_t* ctx, const int32_t* topk_idx, int32_t* hist, void* stream) {

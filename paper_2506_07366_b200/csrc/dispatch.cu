@@ -23,13 +23,17 @@
 #include <atomic>
 
 #include "common.cuh"
+#include "slot_offsets.cuh"
 
 namespace {
+
+using slot_offsets::share_total;
+using slot_offsets::slot_loads_of_expert;
 
 constexpr int kWarpsPerBlock = 8;
 constexpr int kThreads = kWarpsPerBlock * 32;
 constexpr int kMaxE = 256;
-constexpr int kMaxS = 1024;
+constexpr int kMaxS = slot_offsets::kMaxS;
 constexpr int kScanThreads = 1024;
 constexpr int kScanSmemBytes = 100 * 1024;  // staging of the count matrix; two such CTAs still fit one SM
 
@@ -37,57 +41,6 @@ static_assert(kSegPairs == 256, "the count kernels assign one thread to each pai
 static_assert(kMaxS <= 4 * kSegPairs, "count_kernel scans four slots per thread");
 
 constexpr int kDirectMaxSeg = 1024;   // up to this many segments rank_copy sums the counts itself
-
-// Total of the predicted tokens that the copies of an expert were given (slot_share, from
-// moegps_pack_slots); 0 when there is no share table, the prediction gave the expert nothing, or the
-// table is out of range (then the copies take equal parts).
-__device__ __forceinline__ long long share_total(const int32_t* __restrict__ slot_share, int so, int r) {
-  if (!slot_share) return 0;
-  long long tot = 0;
-  for (int rho = 0; rho < r; ++rho) {
-    const int v = slot_share[so + rho];
-    if (v < 0) return 0;
-    tot += v;
-  }
-  return tot > 0x7fffffffll ? 0 : tot;
-}
-
-// Rows reserved for the replicas of expert `e` (loads rounded up to A) -> padded[slot].
-// Replica rho takes ranks floor(rho n/r) .. floor((rho+1) n/r) - 1, or, with a share table, ranks
-// floor(n c_rho / c) .. floor(n c_{rho+1} / c) - 1 with c_rho the shares of the copies before it.
-__device__ __forceinline__ void slot_loads_of_expert(int e, int S, int A, const int32_t* __restrict__ hist,
-                                                     const int32_t* __restrict__ replicas,
-                                                     const int32_t* __restrict__ slot_off,
-                                                     const int32_t* __restrict__ slot_share, int32_t* padded,
-                                                     int32_t* status) {
-  const long long n = hist[e];
-  const int r = replicas[e];
-  const int so = slot_off[e];
-  if (r < 1 || so < 0 || so + r > S || n < 0) {
-    moegps_report(status, MOEGPS_ERR_BAD_INDEX, e);
-    return;
-  }
-  const long long tot = share_total(slot_share, so, r);
-  if (tot > 0) {
-    long long cum = 0;
-    int prev = 0;
-    for (int rho = 0; rho < r; ++rho) {
-      cum += slot_share[so + rho];
-      const int start = (int)((n * cum) / tot);      // n, cum < 2^31
-      padded[so + rho] = (start - prev + A - 1) / A * A;
-      prev = start;
-    }
-    return;
-  }
-  // floor(rho n / r) = rho q + floor(rho m / r) with n = q r + m: one division, then 32-bit work
-  const int q = (int)(n / r), m = (int)(n - (long long)q * r);
-  int prev = 0;
-  for (int rho = 1; rho <= r; ++rho) {
-    const int start = rho * q + (rho * m) / r;     // rho, m < r <= 1024
-    padded[so + rho - 1] = (start - prev + A - 1) / A * A;
-    prev = start;
-  }
-}
 
 // Short pair lists: counts only, stored expert-major; CTA 0 also builds slot_row_off.
 __global__ void __launch_bounds__(kSegPairs)
@@ -98,7 +51,7 @@ count_kernel(const int32_t* __restrict__ topk_idx, int64_t R, int E, int S, int 
   __shared__ int32_t cnt[kMaxE];
   __shared__ int32_t padded[kMaxS];
   __shared__ int32_t warp_tot[kSegPairs / 32];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x, lane = tid & 31;
   const int seg = blockIdx.x;
   // padding rows keep -1: fill everything, occupied rows are overwritten by rank_copy
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + tid; i < Rcap; i += (int64_t)gridDim.x * blockDim.x)
@@ -124,36 +77,8 @@ count_kernel(const int32_t* __restrict__ topk_idx, int64_t R, int E, int S, int 
   if (blockIdx.x != 0) return;
 
   // ---- CTA 0: slot row offsets (independent of the counts) ----
-  for (int s = tid; s < S; s += kSegPairs) padded[s] = 0;
-  __syncthreads();
-  for (int e = tid; e < E; e += kSegPairs) slot_loads_of_expert(e, S, A, hist, replicas, slot_off, slot_share, padded, status);
-  __syncthreads();
-  // slot starts are multiples of A, so the offsets are a plain prefix sum of the padded loads;
-  // thread t owns slots 4t .. 4t+3 (S <= 1024 = 4 * 256)
-  int v[4], sum = 0;
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int s = 4 * tid + i;
-    v[i] = s < S ? padded[s] : 0;
-    sum += v[i];
-  }
-  int incl = sum;
-#pragma unroll
-  for (int d = 1; d < 32; d <<= 1) {
-    const int o = __shfl_up_sync(0xffffffffu, incl, d);
-    if (lane >= d) incl += o;
-  }
-  if (lane == 31) warp_tot[warp] = incl;
-  __syncthreads();
-  int run = incl - sum;
-  for (int wv = 0; wv < warp; ++wv) run += warp_tot[wv];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int s = 4 * tid + i;
-    run += v[i];
-    if (s < S) slot_row_off[s + 1] = run;
-  }
-  if (tid == 0) slot_row_off[0] = 0;
+  slot_offsets::build_slot_row_off<kSegPairs>(E, S, A, hist, replicas, slot_off, slot_share, padded, warp_tot,
+                                              slot_row_off, status);
 }
 
 __global__ void __launch_bounds__(kScanThreads)
@@ -284,6 +209,81 @@ count_scan_kernel(const int32_t* __restrict__ topk_idx, int64_t R, int E, int S,
   if (tid == 0) slot_row_off[0] = 0;
 }
 
+// Second half of the ranking kernels: lane j < K holds pair j of token t with its stable rank
+// (my_rank, -1 if the expert index was out of range).  Replica, slot and row follow in integer
+// arithmetic; then the warp reads the token row once (128-bit loads) and writes it to its K rows.
+__device__ __forceinline__ void place_and_copy(const uint4* __restrict__ x, int t, int K, int chunks, int S, int64_t Rcap,
+                                               int my_e, int my_rank, const int32_t* __restrict__ hist,
+                                               const int32_t* __restrict__ replicas,
+                                               const int32_t* __restrict__ slot_off,
+                                               const int32_t* __restrict__ slot_share,
+                                               const int32_t* __restrict__ slot_row_off,
+                                               int32_t* __restrict__ pair_row, int32_t* __restrict__ row_pair,
+                                               uint4* __restrict__ xp, int32_t* __restrict__ status) {
+  const int lane = threadIdx.x & 31;
+  // ---- replica, slot, row (lane j for pair j) ----
+  int row = -1;
+  if (lane < K && my_rank >= 0) {
+    const long long n = hist[my_e];
+    const int r = replicas[my_e];
+    if (n <= 0 || r < 1 || my_rank >= n) {
+      moegps_report(status, MOEGPS_ERR_HIST_MISMATCH, my_e);
+    } else {
+      const int so = slot_off[my_e];
+      int rho, start;
+      const long long tot = (so >= 0 && so + r <= S) ? share_total(slot_share, so, r) : 0;
+      if (tot > 0) {                                                   // copies take parts in proportion to their shares
+        long long cum = 0;
+        int end = 0;
+        start = 0;
+        for (rho = 0; rho < r - 1; ++rho) {
+          cum += slot_share[so + rho];
+          end = (int)((n * cum) / tot);
+          if (my_rank < end) break;
+          start = end;
+        }
+      } else {
+        rho = (int)((((long long)my_rank + 1) * r - 1) / n);           // replica whose range holds the rank
+        start = (int)(((long long)rho * n) / r);
+      }
+      const int slot = so + rho;
+      const long long rr = (slot >= 0 && slot < S) ? (long long)slot_row_off[slot] + (my_rank - start) : -1;
+      if (rr < 0 || rr >= Rcap) {
+        moegps_report(status, MOEGPS_ERR_BAD_INDEX, t);
+      } else {
+        row = (int)rr;
+        pair_row[(int64_t)t * K + lane] = row;
+        row_pair[row] = (int32_t)((int64_t)t * K + lane);
+      }
+    }
+  }
+  long long dst[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int rj = __shfl_sync(0xffffffffu, row, j);
+    dst[j] = (j < K && rj >= 0) ? (long long)rj * chunks : -1;
+  }
+  // ---- row moves ----
+  const uint4* src = x + (int64_t)t * chunks;
+  int c = lane;
+  for (; c + 96 < chunks; c += 128) {                      // four 16-byte loads in flight per lane
+    const uint4 v0 = src[c], v1 = src[c + 32], v2 = src[c + 64], v3 = src[c + 96];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (dst[j] >= 0) {
+        uint4* d = xp + dst[j];
+        d[c] = v0; d[c + 32] = v1; d[c + 64] = v2; d[c + 96] = v3;
+      }
+    }
+  }
+  for (; c < chunks; c += 32) {
+    const uint4 vv = src[c];
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      if (dst[j] >= 0) xp[dst[j] + c] = vv;
+  }
+}
+
 // kDirect: `seg_base` holds the raw counts expert-major ([E][nseg]) and the warp sums the expert's
 // row up to its segment itself; otherwise it holds the scanned matrix ([nseg][E]).
 template <bool kDirect>
@@ -350,67 +350,76 @@ rank_copy_kernel(const uint4* __restrict__ x, int T, int K, int chunks /* D*2/16
       if (lane == j) my_rank = (my_e >= 0 && my_e < E) ? my_base + rank : -1;
     }
   }
-  // ---- replica, slot, row (lane j for pair j) ----
-  int row = -1;
-  if (lane < K && my_rank >= 0) {
-    const long long n = hist[my_e];
-    const int r = replicas[my_e];
-    if (n <= 0 || r < 1 || my_rank >= n) {
-      moegps_report(status, MOEGPS_ERR_HIST_MISMATCH, my_e);
-    } else {
-      const int so = slot_off[my_e];
-      int rho, start;
-      const long long tot = (so >= 0 && so + r <= S) ? share_total(slot_share, so, r) : 0;
-      if (tot > 0) {                                                   // copies take parts in proportion to their shares
-        long long cum = 0;
-        int end = 0;
-        start = 0;
-        for (rho = 0; rho < r - 1; ++rho) {
-          cum += slot_share[so + rho];
-          end = (int)((n * cum) / tot);
-          if (my_rank < end) break;
-          start = end;
-        }
-      } else {
-        rho = (int)((((long long)my_rank + 1) * r - 1) / n);           // replica whose range holds the rank
-        start = (int)(((long long)rho * n) / r);
-      }
-      const int slot = so + rho;
-      const long long rr = (slot >= 0 && slot < S) ? (long long)slot_row_off[slot] + (my_rank - start) : -1;
-      if (rr < 0 || rr >= Rcap) {
-        moegps_report(status, MOEGPS_ERR_BAD_INDEX, t);
-      } else {
-        row = (int)rr;
-        pair_row[(int64_t)t * K + lane] = row;
-        row_pair[row] = (int32_t)((int64_t)t * K + lane);
+  place_and_copy(x, t, K, chunks, S, Rcap, my_e, my_rank, hist, replicas, slot_off, slot_share, slot_row_off, pair_row,
+                 row_pair, xp, status);
+}
+
+// Dispatch after moegps_route_prepare: the count matrix (one column per router CTA, i.e. per
+// `rows_per` consecutive tokens, expert-major) and the slot row offsets exist already, so this single
+// kernel ranks, places and copies.  One warp per token: the stable rank of a pair = its expert's
+// counts over the earlier columns (a coalesced read by the warp) + the same-expert pairs of the
+// earlier tokens of its own column (the K experts of one token are distinct, so its own pairs never
+// count).  The first S blocks also mark the padding rows of one slot each with -1.
+__global__ void __launch_bounds__(kThreads)
+rank_copy_prepared_kernel(const uint4* __restrict__ x, int T, int K, int chunks, const int32_t* __restrict__ topk_idx,
+                          int E, int S, int64_t Rcap, const int32_t* __restrict__ seg_cnt, int nsub, int rows_per,
+                          const int32_t* __restrict__ hist, const int32_t* __restrict__ replicas,
+                          const int32_t* __restrict__ slot_off, const int32_t* __restrict__ slot_row_off,
+                          int32_t* __restrict__ pair_row, int32_t* __restrict__ row_pair, uint4* __restrict__ xp,
+                          int32_t* __restrict__ status) {
+  __shared__ int pad_begin, pad_end;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  // ---- padding rows of slots blockIdx.x, blockIdx.x + gridDim.x, ... ----
+  for (int b = blockIdx.x; b < S; b += gridDim.x) {
+    if (threadIdx.x == 0) { pad_begin = 0; pad_end = 0; }
+    __syncthreads();
+    const int e = threadIdx.x;                       // blockDim = 256 >= E: the thread of the slot's expert answers
+    if (e < E) {
+      const int so = slot_off[e], r = replicas[e];
+      if (r >= 1 && so <= b && b < so + r) {
+        const long long n = hist[e];
+        const int rho = b - so;
+        const int load = (int)(((long long)(rho + 1) * n) / r - ((long long)rho * n) / r);
+        pad_begin = slot_row_off[b] + load;
+        pad_end = slot_row_off[b + 1];
       }
     }
+    __syncthreads();
+    for (int row = pad_begin + threadIdx.x; row < pad_end; row += kThreads)
+      if (row >= 0 && row < Rcap) row_pair[row] = -1;
+    __syncthreads();
   }
-  long long dst[8];
+  // ---- and the rows behind the last slot ----
+  for (int64_t row = (int64_t)slot_row_off[S] + (int64_t)blockIdx.x * kThreads + threadIdx.x; row < Rcap;
+       row += (int64_t)gridDim.x * kThreads)
+    if (row >= 0) row_pair[row] = -1;
+  const int t = blockIdx.x * kWarpsPerBlock + warp;
+  if (t >= T) return;
+  // ---- ranks of this token's K pairs (lane j ends up holding pair j) ----
+  const int sub = t / rows_per;
+  const int64_t q_begin = (int64_t)sub * rows_per * K, q_end = (int64_t)t * K;
+  int my_e = -1, my_rank = -1;
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
-    const int rj = __shfl_sync(0xffffffffu, row, j);
-    dst[j] = (j < K && rj >= 0) ? (long long)rj * chunks : -1;
-  }
-  // ---- row moves ----
-  const uint4* src = x + (int64_t)t * chunks;
-  int c = lane;
-  for (; c + 96 < chunks; c += 128) {                      // four 16-byte loads in flight per lane
-    const uint4 v0 = src[c], v1 = src[c + 32], v2 = src[c + 64], v3 = src[c + 96];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      if (dst[j] >= 0) {
-        uint4* d = xp + dst[j];
-        d[c] = v0; d[c + 32] = v1; d[c + 64] = v2; d[c + 96] = v3;
+    if (j < K) {
+      const int e = topk_idx[(int64_t)t * K + j];
+      const bool valid = e >= 0 && e < E;
+      int c = 0;
+      for (int64_t q = q_begin + lane; q < q_end; q += 32) c += topk_idx[q] == e ? 1 : 0;   // earlier tokens of this column
+      if (valid) {                                                                          // earlier columns
+        const int32_t* cnt_row = seg_cnt + (int64_t)e * nsub;
+        for (int g = lane; g < sub; g += 32) c += cnt_row[g];
+      }
+      const int rank = __reduce_add_sync(0xffffffffu, c);
+      if (lane == j) {
+        my_e = e;
+        my_rank = valid ? rank : -1;
+        if (!valid) moegps_report(status, MOEGPS_ERR_BAD_INDEX, t);
       }
     }
   }
-  for (; c < chunks; c += 32) {
-    const uint4 vv = src[c];
-#pragma unroll
-    for (int j = 0; j < 8; ++j)
-      if (dst[j] >= 0) xp[dst[j] + c] = vv;
-  }
+  place_and_copy(x, t, K, chunks, S, Rcap, my_e, my_rank, hist, replicas, slot_off, nullptr, slot_row_off, pair_row,
+                 row_pair, xp, status);
 }
 
 }  // namespace
@@ -458,6 +467,22 @@ int moegps_launch_dispatch(moegps_ctx* ctx, const void* x, const int32_t* topk_i
         static_cast<const uint4*>(x), s.T, s.K, s.D / 8, topk_idx, R, s.E, s.S, Rcap, seg, nseg, hist, replicas, slot_off,
         slot_share, slot_row_off, pair_row, row_pair, static_cast<uint4*>(xp), ctx->d_status);
   }
+  MOEGPS_AFTER_LAUNCH(ctx);
+  return MOEGPS_OK;
+}
+
+int moegps_launch_dispatch_prepared(moegps_ctx* ctx, const void* x, const int32_t* topk_idx, const int32_t* hist,
+                                    const int32_t* replicas, const int32_t* slot_off,
+                                    const int32_t* slot_row_off, int32_t* row_pair, int32_t* pair_row, void* xp,
+                                    const void* workspace, cudaStream_t st) {
+  const moegps_shape_t& s = ctx->shape;
+  const int rows_per = moegps_route_rows_per_cta(ctx);
+  const int nsub = (s.T + 127) / 128 * (128 / rows_per);
+  const int tblocks = (s.T + kWarpsPerBlock - 1) / kWarpsPerBlock;
+  rank_copy_prepared_kernel<<<tblocks, kThreads, 0, st>>>(
+      static_cast<const uint4*>(x), s.T, s.K, s.D / 8, topk_idx, s.E, s.S, moegps_rcap_of(s),
+      static_cast<const int32_t*>(workspace), nsub, rows_per, hist, replicas, slot_off, slot_row_off, pair_row, row_pair,
+      static_cast<uint4*>(xp), ctx->d_status);
   MOEGPS_AFTER_LAUNCH(ctx);
   return MOEGPS_OK;
 }

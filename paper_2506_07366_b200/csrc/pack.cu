@@ -66,6 +66,15 @@ pack_kernel(const int32_t* __restrict__ pred, const int32_t* __restrict__ home, 
     if (lane < G) l0 += share[e * G + lane];
     if (lane + 32 < G) l1 += share[e * G + lane + 32];
   }
+  {   // the loads are returned as int32: all predicted tokens together must fit
+    long long total = l0 + l1;
+#pragma unroll
+    for (int m = 16; m >= 1; m >>= 1) total += __shfl_xor_sync(0xffffffffu, total, m);
+    if (total > 0x7fffffffll) {
+      if (lane == 0) moegps_report(status, MOEGPS_ERR_BAD_INDEX, E);
+      bad = true;
+    }
+  }
   int iters = 0;
   while (!bad && iters < kMaxIters) {
     // (load, device) packed so that one max finds the hottest / coldest device, lowest index on ties

@@ -21,12 +21,17 @@
 // Selection: L lanes per token select by shuffles (route_epilogue.cuh), L chosen so that the rows the
 // CTA owns occupy all sixteen warps in one pass.  When the caller asks for it, the per-expert token
 // counts (Eq. 1's n_e) are accumulated on the way: every selection bumps a shared-memory counter of
-// its CTA, and each CTA adds its non-zero counters to the global histogram once (integer atomics:
-// deterministic).
+// its CTA; each CTA adds its non-zero counters to accumulators that belong to the context (integer
+// atomics: deterministic) and draws a ticket; the CTA that draws the last one copies the sums to the
+// caller's histogram and leaves accumulators and ticket at zero for the next call - no memset, no
+// second kernel.  In the fused form (moegps_route_prepare) every CTA also stores its counters as one
+// column of the count matrix that dispatch ranks pairs with, and the last CTA derives the slot row
+// offsets from the finished histogram, so that dispatch is a single launch.
 // Warp roles in the main loop: warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
 // warps 2..5 = drain.  Every mbarrier wait is bounded.
 #include "common.cuh"
 #include "route_epilogue.cuh"
+#include "slot_offsets.cuh"
 #include "sm100.cuh"
 
 bool moegps_make_tmap_2d(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
@@ -160,8 +165,10 @@ __global__ void __launch_bounds__(kThreads, 1)
 route_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
              const RouteParams p, const float* __restrict__ bias, int32_t* __restrict__ topk_idx,
              float* __restrict__ topk_w, float* __restrict__ logits_out, int32_t* __restrict__ hist,
-             int32_t* __restrict__ status) {
+             int32_t* __restrict__ acc /* context-owned: [256] sums + ticket at [256] */,
+             const moegps_route_fused fused, int S, int row_align, int32_t* __restrict__ status) {
   __shared__ int32_t cta_hist[256];       // this CTA's share of the histogram (used when hist != nullptr)
+  __shared__ int32_t s_last;
   __shared__ float s_bias[256];           // fetched while the stream runs
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -302,24 +309,64 @@ route_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     if (topk_idx) select_stage(p, partial, rows_per, t0, topk_idx, topk_w, hist ? cta_hist : nullptr, false);
   }
   __syncthreads();
-  if (hist) {
-    for (int e = threadIdx.x; e < p.E; e += kThreads) {
-      const int c = cta_hist[e];
-      if (c) atomicAdd(&hist[e], c);
-    }
-  }
-  if (warp == 1) {
+  if (warp == 1) {                // TMEM is no longer needed; release it before the tail below
     tc_fence_after_sync();
     tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+  }
+  if (hist) {
+    const int n_ctas = (int)(gridDim.x * gridDim.y);
+    const int sub = (int)blockIdx.x * p.ks + (int)rank;          // this CTA's column of the count matrix
+    for (int e = threadIdx.x; e < p.E; e += kThreads) {
+      const int c = cta_hist[e];
+      if (fused.seg_cnt) fused.seg_cnt[(int64_t)e * n_ctas + sub] = c;
+      if (c) atomicAdd(&acc[e], c);
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = atomicAdd(&acc[256], 1) == n_ctas - 1;
+    __syncthreads();
+    if (s_last) {                 // every CTA's sums are in: publish them and leave the accumulators at zero
+      __threadfence();
+      for (int e = threadIdx.x; e < p.E; e += kThreads) {
+        const int h = atomicExch(&acc[e], 0);
+        hist[e] = h;
+        cta_hist[e] = h;          // (re-used as the finished histogram for the offsets below)
+      }
+      if (threadIdx.x == 0) acc[256] = 0;
+      if (fused.seg_cnt) {
+        // slot row offsets of the dispatch step (they depend on the finished histogram only);
+        // the ring memory is free by now and serves as scratch
+        int32_t* padded = reinterpret_cast<int32_t*>(smem);
+        int32_t* warp_tot = padded + slot_offsets::kMaxS;
+        __syncthreads();
+        slot_offsets::build_slot_row_off<kThreads>(p.E, S, row_align, cta_hist, fused.replicas, fused.slot_off,
+                                                   nullptr, padded, warp_tot, fused.slot_row_off, status);
+      }
+    }
   }
 }
 
 }  // namespace
 
-int moegps_launch_route(moegps_ctx* ctx, const void* x, const void* wr, const float* bias, int32_t* topk_idx,
-                        float* topk_w, float* logits_out, int32_t* hist, cudaStream_t st) {
+namespace {
+// How the model dimension is split: until the grid covers most of the chip (cluster size <= 8, a
+// power of two so that 128 rows divide evenly, and every slice keeps at least 4 K blocks).
+int route_split(const moegps_ctx* ctx) {
   const moegps_shape_t& s = ctx->shape;
-  if (hist) MOEGPS_CUDA_TRY(ctx, cudaMemsetAsync(hist, 0, sizeof(int32_t) * s.E, st));
+  const int nkb = (s.D + BK - 1) / BK;
+  const int tiles = (s.T + BM - 1) / BM;
+  int ks = 1;
+  while (ks < 8 && tiles * ks * 2 <= ctx->sm_count + ctx->sm_count / 4 && nkb / (ks * 2) >= 4) ks *= 2;
+  return ks;
+}
+}  // namespace
+
+int moegps_route_rows_per_cta(const moegps_ctx* ctx) { return BM / route_split(ctx); }
+
+int moegps_launch_route(moegps_ctx* ctx, const void* x, const void* wr, const float* bias, int32_t* topk_idx,
+                        float* topk_w, float* logits_out, int32_t* hist, const moegps_route_fused* fused,
+                        cudaStream_t st) {
+  const moegps_shape_t& s = ctx->shape;
   RouteParams p;
   p.T = s.T; p.D = s.D; p.E = s.E; p.K = s.K; p.gate_mode = s.gate_mode;
   p.e_pad = (s.E + 15) / 16 * 16;
@@ -328,10 +375,7 @@ int moegps_launch_route(moegps_ctx* ctx, const void* x, const void* wr, const fl
   if (p.stages > 10) p.stages = 10;
   const int nkb = (s.D + BK - 1) / BK;
   const int tiles = (s.T + BM - 1) / BM;
-  // split the model dimension until the grid covers most of the chip (cluster size <= 8, a power
-  // of two so that 128 rows divide evenly, and every slice keeps at least 4 K blocks)
-  int ks = 1;
-  while (ks < 8 && tiles * ks * 2 <= ctx->sm_count + ctx->sm_count / 4 && nkb / (ks * 2) >= 4) ks *= 2;
+  const int ks = route_split(ctx);
   p.ks = ks;
   p.kb_per_cta = (nkb + ks - 1) / ks;
   if (p.stages > p.kb_per_cta) p.stages = p.kb_per_cta < 2 ? 2 : p.kb_per_cta;
@@ -374,8 +418,10 @@ int moegps_launch_route(moegps_ctx* ctx, const void* x, const void* wr, const fl
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  const moegps_route_fused none = {nullptr, nullptr, nullptr, nullptr};
   cudaError_t e = cudaLaunchKernelEx(&cfg, route_kernel, ctx->tm_rx, ctx->tm_rw, p, bias, topk_idx, topk_w,
-                                     logits_out, hist, ctx->d_status);
+                                     logits_out, hist, ctx->d_route_acc, fused ? *fused : none, (int)s.S,
+                                     (int)s.row_align, ctx->d_status);
   ctx->launches += 1;
   if (e != cudaSuccess) {
     ctx->last_cuda_error = (int)e;

@@ -43,7 +43,7 @@ HAND = [
     ([5, 0], [0, 1], [2, 2], 0), ([4, 4, 0, 0], [0, 1, 2, 3], [2, 2, 2, 2], 0), ([3, 3, 1], [0, 0, 0], [3, 3], 0),
     ([7, 2], [0, 0], [2], 0), ([3, 4], [0, 1], [2, 2], 0), ([1000, 10, 10, 10], [0, 1, 2, 3], [4] * 4, 1),
     ([1000, 10, 10, 10], [0, 1, 2, 3], [4] * 4, 2), ([1000, 10, 10, 10], [0, 1, 2, 3], [1] * 4, 0),
-    ([100], [0], [1, 1, 1], 0), ([0, 0, 0], [2, 1, 0], [1, 1, 1], 0), ([2 ** 31 - 1, 5], [0, 1], [2, 2], 0),
+    ([100], [0], [1, 1, 1], 0), ([0, 0, 0], [2, 1, 0], [1, 1, 1], 0), ([2 ** 31 - 6, 5], [0, 1], [2, 2], 0),
 ]
 
 
@@ -73,6 +73,8 @@ def test_pack_reports_bad_inputs_without_faulting():
     ctx, placed, share, load, iters = run_pack(np.array([5, 5, 5]), [0, 7, 1], [2, 2], 0)      # home out of range
     assert ctx.status() == binding.ERR_BAD_INDEX and iters == 0
     ctx, placed, share, load, iters = run_pack(np.array([5, 5, 5]), [0, 0, 0], [2, 3], 0)      # device 0 over-full
+    assert ctx.status() == binding.ERR_BAD_INDEX and iters == 0
+    ctx, placed, share, load, iters = run_pack(np.array([2 ** 31 - 1, 5]), [0, 1], [2, 2], 0)  # loads would not fit int32
     assert ctx.status() == binding.ERR_BAD_INDEX and iters == 0
     ctx = binding.Context(binding.Shape(8, 64, 64, 4, 1, 4, 0, 1))
     with pytest.raises(binding.MoegpsError) as ei:                                                # too many devices

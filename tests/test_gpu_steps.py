@@ -225,6 +225,69 @@ def test_dispatch(T, D, E, K, S, A, skew):
     assert (got_xp[~occ] == 0x5A5A).all()          # padding rows are not written
 
 
+FUSED_CASES = [
+    # workload, A          (clusters of 1, 2, 4 and 8 router CTAs per tile; E from 5 to 256; K from 1 to 8; ragged T)
+    (small("tiny", T=256, D=512), 128), (small("mixtral", T=1024, D=4096), 16), (small("mixtral", T=2944, D=2048), 1),
+    (small("many_expert", T=1000, D=4096), 16), (small("fine_grained", T=515, D=1024), 16),
+    (small("fine_grained", T=130, D=4096, S=300), 128), (small("tiny", T=65, D=64, E=5, K=5, S=9), 4),
+    (small("tiny", T=40, D=64, E=33, K=1, S=40, gate_mode=1), 8), (small("mixtral_skew", T=16384 + 77, D=256), 16),
+]
+
+
+@pytest.mark.parametrize("w,A", FUSED_CASES, ids=lambda v: v if isinstance(v, int) else f"{v.name}-T{v.T}-D{v.D}-E{v.E}-K{v.K}")
+def test_route_prepare_and_dispatch_prepared_equal_the_separate_calls_and_the_oracle(w, A):
+    """The two-launch form (router also produces the counts and offsets dispatch needs) against the
+    four-launch form, bit for bit, and against the oracle; twice in a row with different batches,
+    because the router's accumulators live in the context and must be back at zero after every call."""
+    wr, bias = wl.router(w, "cpu")
+    shape = binding.Shape(w.T, w.D, 64, w.E, w.K, w.S, w.gate_mode, A)
+    ctx = binding.Context(shape)
+    wrd, bd = wr.to(DEV), bias.to(DEV)
+    ws_a = torch.full((binding.workspace_bytes(shape),), 0xEE, dtype=torch.uint8, device=DEV)
+    ws_b = torch.full((binding.workspace_bytes(shape),), 0xEE, dtype=torch.uint8, device=DEV)
+    for call in range(2):
+        x, _ = hz.screened_activations(w.scaled(number=w.number + 13 * call), wr, bias)
+        xd = x.to(DEV)
+        ref_idx, ref_w, _ = oracle.route(hz.bits(x), hz.bits(wr), bias.numpy(), w.K, w.gate_mode)
+        ref_hist = oracle.histogram(ref_idx, w.E)
+        pred = np.maximum(0, np.round(ref_hist * (1 + 0.2 * np.random.default_rng(call).normal(size=w.E)))).astype(np.int64)
+        rep_ref, so_ref, _, _ = oracle.plan(pred, w.S)
+        rep, so = i32(rep_ref), i32(so_ref)
+        # separate calls
+        idx_a, wt_a, hist_a = poison_i32(w.T, w.K), torch.full((w.T, w.K), float("nan"), device=DEV), poison_i32(w.E)
+        sro_a, rp_a, pr_a = poison_i32(w.S + 1), poison_i32(shape.Rcap), poison_i32(w.T, w.K)
+        xp_a = torch.full((shape.Rcap, w.D), 0x5A5A, dtype=torch.int16, device=DEV).view(torch.bfloat16)
+        ctx.route_histogram(xd, wrd, bd, idx_a, wt_a, hist_a)
+        ctx.dispatch(xd, idx_a, hist_a, rep, so, sro_a, rp_a, pr_a, xp_a, ws_a)
+        # fused calls
+        idx_b, wt_b, hist_b = poison_i32(w.T, w.K), torch.full((w.T, w.K), float("nan"), device=DEV), poison_i32(w.E)
+        sro_b, rp_b, pr_b = poison_i32(w.S + 1), poison_i32(shape.Rcap), poison_i32(w.T, w.K)
+        xp_b = torch.full((shape.Rcap, w.D), 0x5A5A, dtype=torch.int16, device=DEV).view(torch.bfloat16)
+        ctx.route_prepare(xd, wrd, bd, rep, so, idx_b, wt_b, hist_b, sro_b, ws_b)
+        ctx.dispatch_prepared(xd, idx_b, hist_b, rep, so, sro_b, rp_b, pr_b, xp_b, ws_b)
+        ctx.check_status()
+        for a, b, what in ((idx_a, idx_b, "topk_idx"), (wt_a, wt_b, "topk_w"), (hist_a, hist_b, "hist"),
+                           (sro_a, sro_b, "slot_row_off"), (rp_a, rp_b, "row_pair"), (pr_a, pr_b, "pair_row")):
+            assert torch.equal(a, b), (call, what)
+        assert torch.equal(xp_a.view(torch.int16), xp_b.view(torch.int16)), (call, "xp")
+        sro_ref, rp_ref, pr_ref, _ = oracle.dispatch(None, ref_idx, ref_hist, rep_ref, so_ref, w.S, A)
+        assert np.array_equal(idx_b.cpu().numpy(), ref_idx) and np.array_equal(hist_b.cpu().numpy(), ref_hist)
+        assert np.array_equal(sro_b.cpu().numpy(), sro_ref)
+        assert np.array_equal(rp_b.cpu().numpy(), rp_ref) and np.array_equal(pr_b.cpu().numpy(), pr_ref)
+
+
+def test_route_prepare_without_tokens():
+    shape = binding.Shape(0, 64, 64, 4, 2, 6, 0, 8)
+    ctx = binding.Context(shape)
+    hist, sro = poison_i32(4), poison_i32(7)
+    ws = torch.zeros(binding.workspace_bytes(shape), dtype=torch.uint8, device=DEV)
+    ctx.route_prepare(torch.zeros(0, 64, dtype=torch.bfloat16, device=DEV), torch.zeros(4, 64, dtype=torch.bfloat16, device=DEV),
+                      None, i32([2, 2, 1, 1]), i32([0, 2, 4, 5, 6]), torch.zeros(0, 2, dtype=torch.int32, device=DEV),
+                      torch.zeros(0, 2, dtype=torch.float32, device=DEV), hist, sro, ws)
+    ctx.check_status()
+    assert hist.tolist() == [0] * 4 and sro.tolist() == [0] * 7
+
+
 def test_dispatch_detects_hist_mismatch():
     T, D, E, K, S = 64, 64, 4, 2, 6
     rng = np.random.default_rng(3)
