@@ -119,7 +119,9 @@ MOEGPS_API int moegps_route_histogram(moegps_ctx_t* ctx, const void* x, const vo
  * route_prepare: x, w_router, bias, topk_idx, topk_w, hist as in moegps_route_histogram; replicas,
  * slot_off from moegps_plan; slot_row_off: int32 [S+1] (output); workspace:
  * moegps_workspace_bytes(shape) bytes, written here and read by dispatch_prepared (the layout is
- * private to the library: pass the same buffer, untouched, on the same stream).
+ * private to the library: pass the same buffer, untouched, on the same stream).  Like
+ * moegps_route_histogram it sums the counts in accumulators of the context: calls of one context
+ * must not overlap on the GPU.
  * dispatch_prepared: arguments as moegps_dispatch, except that slot_row_off and workspace are inputs. */
 MOEGPS_API int moegps_route_prepare(moegps_ctx_t* ctx, const void* x, const void* w_router, const float* bias,
                                     const int32_t* replicas, const int32_t* slot_off, int32_t* topk_idx,
