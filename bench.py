@@ -236,9 +236,8 @@ class Bench:
     def step(self, record: bool):
         L, c, w = self.layer, self.ctx, self.w
         c.plan(self.pred_dev, w.S, L.replicas, L.slot_off, L.slot_expert, L.bound)
-        # route + histogram + what dispatch needs (counts, slot row offsets) in one kernel, dispatch in one
-        c.route_prepare(self.x, self.wr, self.bias, L.replicas, L.slot_off, L.topk_idx, L.topk_w, L.hist,
-                        L.slot_row_off, L.workspace)
+        # route + histogram + the counts dispatch ranks with in one kernel, dispatch in one
+        c.route_prepare(self.x, self.wr, self.bias, L.topk_idx, L.topk_w, L.hist, L.workspace)
         c.dispatch_prepared(self.x, L.topk_idx, L.hist, L.replicas, L.slot_off, L.slot_row_off, L.row_pair,
                             L.pair_row, L.xp, L.workspace)
         stream = torch.cuda.current_stream()
@@ -343,8 +342,8 @@ class Bench:
             ("dispatch", lambda: c.dispatch(self.x, L.topk_idx, L.hist, L.replicas, L.slot_off, L.slot_row_off,
                                             L.row_pair, L.pair_row, L.xp, L.workspace),
              2.0 * T * D + 2.0 * R * D + 12.0 * R, None),
-            ("route_prepare", lambda: c.route_prepare(self.x, self.wr, self.bias, L.replicas, L.slot_off, L.topk_idx,
-                                                      L.topk_w, L.hist, L.slot_row_off, L.workspace),
+            ("route_prepare", lambda: c.route_prepare(self.x, self.wr, self.bias, L.topk_idx, L.topk_w, L.hist,
+                                                      L.workspace),
              2.0 * T * D + 2.0 * E * D + 8.0 * T * K, 2.0 * T * D * E),
             ("dispatch_prepared", lambda: c.dispatch_prepared(self.x, L.topk_idx, L.hist, L.replicas, L.slot_off,
                                                               L.slot_row_off, L.row_pair, L.pair_row, L.xp,

@@ -112,24 +112,22 @@ MOEGPS_API int moegps_route_histogram(moegps_ctx_t* ctx, const void* x, const vo
 /* route_prepare + dispatch_prepared - the same results as moegps_route_histogram followed by
  * moegps_dispatch, in two launches instead of four.  The router's epilogue already holds, per CTA,
  * the per-expert counts of the token rows that CTA owns; route_prepare stores them as the columns of
- * the count matrix that dispatch ranks pairs with (into `workspace`), and the CTA that finishes last
- * derives slot_row_off from the finished histogram and the plan; dispatch_prepared then only ranks,
- * places and copies (and marks padding rows of row_pair with -1).  Copies of an expert share its
- * pairs evenly (as in moegps_dispatch).  Bit-identical to the separate calls.
- * route_prepare: x, w_router, bias, topk_idx, topk_w, hist as in moegps_route_histogram; replicas,
- * slot_off from moegps_plan; slot_row_off: int32 [S+1] (output); workspace:
+ * the count matrix that dispatch ranks pairs with (into `workspace`); dispatch_prepared derives
+ * slot_row_off from the finished histogram and the plan, ranks, places and copies (and marks padding
+ * rows of row_pair with -1).  Copies of an expert share its pairs evenly (as in moegps_dispatch).
+ * Bit-identical to the separate calls.
+ * route_prepare: x, w_router, bias, topk_idx, topk_w, hist as in moegps_route_histogram; workspace:
  * moegps_workspace_bytes(shape) bytes, written here and read by dispatch_prepared (the layout is
  * private to the library: pass the same buffer, untouched, on the same stream).  Like
  * moegps_route_histogram it sums the counts in accumulators of the context: calls of one context
  * must not overlap on the GPU.
- * dispatch_prepared: arguments as moegps_dispatch, except that slot_row_off and workspace are inputs. */
+ * dispatch_prepared: arguments as moegps_dispatch, except that workspace is an input. */
 MOEGPS_API int moegps_route_prepare(moegps_ctx_t* ctx, const void* x, const void* w_router, const float* bias,
-                                    const int32_t* replicas, const int32_t* slot_off, int32_t* topk_idx,
-                                    float* topk_w, int32_t* hist, int32_t* slot_row_off, void* workspace,
+                                    int32_t* topk_idx, float* topk_w, int32_t* hist, void* workspace,
                                     void* stream);
 MOEGPS_API int moegps_dispatch_prepared(moegps_ctx_t* ctx, const void* x, const int32_t* topk_idx,
                                         const int32_t* hist, const int32_t* replicas, const int32_t* slot_off,
-                                        const int32_t* slot_row_off, int32_t* row_pair, int32_t* pair_row,
+                                        int32_t* slot_row_off, int32_t* row_pair, int32_t* pair_row,
                                         void* xp, const void* workspace, void* stream);
 
 /* Debug companion of moegps_route: also stores the fp32 logits (fp32 [T,E]) the selection was made on. */

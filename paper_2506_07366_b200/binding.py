@@ -95,7 +95,7 @@ def _lib():
         "moegps_workspace_bytes": (ctypes.c_size_t, [ctypes.POINTER(moegps_shape_t)]),
         "moegps_route": (ctypes.c_int, [vp] * 7),
         "moegps_route_histogram": (ctypes.c_int, [vp] * 8),
-        "moegps_route_prepare": (ctypes.c_int, [vp] * 12),
+        "moegps_route_prepare": (ctypes.c_int, [vp] * 9),
         "moegps_dispatch_prepared": (ctypes.c_int, [vp] * 12),
         "moegps_route_logits": (ctypes.c_int, [vp] * 6),
         "moegps_histogram": (ctypes.c_int, [vp] * 4),
@@ -201,8 +201,7 @@ class Context:
             _ptr(topk_w, torch.float32, (s.T, s.K), "topk_w"),
             _ptr(hist, torch.int32, (s.E,), "hist"), _stream(stream)), "moegps_route_histogram")
 
-    def route_prepare(self, x, w_router, bias, replicas, slot_off, topk_idx, topk_w, hist, slot_row_off, workspace,
-                      stream=None):
+    def route_prepare(self, x, w_router, bias, topk_idx, topk_w, hist, workspace, stream=None):
         s = self.shape
         if workspace is None or workspace.numel() * workspace.element_size() < workspace_bytes(s):
             raise MoegpsError(ERR_WORKSPACE_TOO_SMALL, "moegps_route_prepare")
@@ -210,12 +209,9 @@ class Context:
             self._h, _ptr(x, torch.bfloat16, (s.T, s.D), "x"),
             _ptr(w_router, torch.bfloat16, (s.E, s.D), "w_router"),
             _ptr(bias, torch.float32, (s.E,), "bias", allow_none=True),
-            _ptr(replicas, torch.int32, (s.E,), "replicas"),
-            _ptr(slot_off, torch.int32, (s.E + 1,), "slot_off"),
             _ptr(topk_idx, torch.int32, (s.T, s.K), "topk_idx"),
             _ptr(topk_w, torch.float32, (s.T, s.K), "topk_w"),
             _ptr(hist, torch.int32, (s.E,), "hist"),
-            _ptr(slot_row_off, torch.int32, (s.S + 1,), "slot_row_off"),
             _ptr(workspace, workspace.dtype, None, "workspace"), _stream(stream)), "moegps_route_prepare")
 
     def dispatch_prepared(self, x, topk_idx, hist, replicas, slot_off, slot_row_off, row_pair, pair_row, xp,

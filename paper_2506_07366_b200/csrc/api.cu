@@ -57,10 +57,10 @@ int moegps_create(moegps_ctx_t** out, const moegps_shape_t* shape, int device) {
   cudaGetDevice(&prev);
   cudaError_t e = cudaSetDevice(device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
-  constexpr size_t kCtxWords = 4 + 256 + 4;      // status word, router accumulators, router ticket
+  constexpr size_t kCtxWords = 4 + 2 * 256;      // status word, router accumulators (64-bit)
   if (e == cudaSuccess) e = cudaMalloc(&ctx->d_status, kCtxWords * sizeof(int32_t));
   if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, kCtxWords * sizeof(int32_t));
-  ctx->d_route_acc = ctx->d_status ? ctx->d_status + 4 : nullptr;
+  ctx->d_route_acc = ctx->d_status ? reinterpret_cast<unsigned long long*>(ctx->d_status + 4) : nullptr;
   cudaSetDevice(prev);
   if (e != cudaSuccess) {
     if (ctx->d_status) cudaFree(ctx->d_status);
@@ -120,28 +120,29 @@ int moegps_route_histogram(moegps_ctx_t* ctx, const void* x, const void* w_route
 }
 
 int moegps_route_prepare(moegps_ctx_t* ctx, const void* x, const void* w_router, const float* bias,
-                         const int32_t* replicas, const int32_t* slot_off, int32_t* topk_idx, float* topk_w,
-                         int32_t* hist, int32_t* slot_row_off, void* workspace, void* stream) {
-  if (!ctx || !all_ok(replicas, slot_off, hist, slot_row_off, workspace)) return MOEGPS_ERR_INVALID_ARG;
+                         int32_t* topk_idx, float* topk_w, int32_t* hist, void* workspace, void* stream) {
+  if (!ctx || !all_ok(hist, workspace)) return MOEGPS_ERR_INVALID_ARG;
   if (int rc = moegps_check_device(ctx)) return rc;
   cudaStream_t st = (cudaStream_t)stream;
-  if (ctx->shape.T == 0) {                          // no tokens: empty histogram, every slot empty
+  if (ctx->shape.T == 0) {                          // no tokens: the histogram is all zero
     MOEGPS_CUDA_TRY(ctx, cudaMemsetAsync(hist, 0, sizeof(int32_t) * ctx->shape.E, st));
-    MOEGPS_CUDA_TRY(ctx, cudaMemsetAsync(slot_row_off, 0, sizeof(int32_t) * (ctx->shape.S + 1), st));
     return MOEGPS_OK;
   }
   if (!all_ok(x, w_router, topk_idx, topk_w)) return MOEGPS_ERR_INVALID_ARG;
   if (bias && (reinterpret_cast<uintptr_t>(bias) & 3u)) return MOEGPS_ERR_INVALID_ARG;
-  const moegps_route_fused fused = {static_cast<int32_t*>(workspace), replicas, slot_off, slot_row_off};
-  return moegps_launch_route(ctx, x, w_router, bias, topk_idx, topk_w, nullptr, hist, &fused, st);
+  return moegps_launch_route(ctx, x, w_router, bias, topk_idx, topk_w, nullptr, hist, static_cast<int32_t*>(workspace),
+                             st);
 }
 
 int moegps_dispatch_prepared(moegps_ctx_t* ctx, const void* x, const int32_t* topk_idx, const int32_t* hist,
-                             const int32_t* replicas, const int32_t* slot_off, const int32_t* slot_row_off,
+                             const int32_t* replicas, const int32_t* slot_off, int32_t* slot_row_off,
                              int32_t* row_pair, int32_t* pair_row, void* xp, const void* workspace, void* stream) {
   if (!ctx || !all_ok(hist, replicas, slot_off, slot_row_off, workspace)) return MOEGPS_ERR_INVALID_ARG;
   if (int rc = moegps_check_device(ctx)) return rc;
-  if (ctx->shape.T == 0) return MOEGPS_OK;          // nothing routed: no row is occupied, no padding exists
+  if (ctx->shape.T == 0) {                          // nothing routed: every slot is empty, no padding exists
+    MOEGPS_CUDA_TRY(ctx, cudaMemsetAsync(slot_row_off, 0, sizeof(int32_t) * (ctx->shape.S + 1), (cudaStream_t)stream));
+    return MOEGPS_OK;
+  }
   if (!all_ok(x, topk_idx, pair_row, xp, row_pair)) return MOEGPS_ERR_INVALID_ARG;
   return moegps_launch_dispatch_prepared(ctx, x, topk_idx, hist, replicas, slot_off, slot_row_off, row_pair, pair_row,
                                          xp, workspace, (cudaStream_t)stream);

@@ -14,7 +14,7 @@ struct moegps_ctx {
   int device;
   int sm_count;
   int32_t* d_status;        // 4 x int32 on the device
-  int32_t* d_route_acc;     // behind it: 256 histogram accumulators of the router + its ticket counter (all zero between calls)
+  unsigned long long* d_route_acc;   // behind it: 256 64-bit histogram accumulators of the router (all zero between calls)
   int64_t launches;         // kernels launched through this context
   int last_cuda_error;
   // cached TMA descriptors of the expert FFN, keyed by the base pointers they were built for
@@ -77,21 +77,15 @@ __device__ __forceinline__ void moegps_report(int32_t* status, int code, int det
 constexpr int kSegPairs = 256;
 
 // Per-step launchers (each validates nothing: the C entry points in api.cu do that).
-// What the router's fused tail needs to prepare the dispatch step (seg_cnt == nullptr: not fused).
-struct moegps_route_fused {
-  int32_t* seg_cnt;              // [E][tiles*KS] per-CTA counts, expert-major
-  const int32_t* replicas;
-  const int32_t* slot_off;
-  int32_t* slot_row_off;
-};
+// seg_cnt != nullptr: the router also stores its per-CTA expert counts, [E][CTAs] expert-major.
 int moegps_launch_route(moegps_ctx* ctx, const void* x, const void* wr, const float* bias,
                         int32_t* topk_idx, float* topk_w, float* logits_out, int32_t* hist,
-                        const moegps_route_fused* fused, cudaStream_t st);
+                        int32_t* seg_cnt, cudaStream_t st);
 // rows of a token tile that one router CTA owns (= 128 / its split of the model dimension)
 int moegps_route_rows_per_cta(const moegps_ctx* ctx);
 int moegps_launch_dispatch_prepared(moegps_ctx* ctx, const void* x, const int32_t* topk_idx, const int32_t* hist,
                                     const int32_t* replicas, const int32_t* slot_off,
-                                    const int32_t* slot_row_off, int32_t* row_pair, int32_t* pair_row, void* xp,
+                                    int32_t* slot_row_off, int32_t* row_pair, int32_t* pair_row, void* xp,
                                     const void* workspace, cudaStream_t st);
 int moegps_launch_histogram(moegps_ctx* ctx, const int32_t* topk_idx, int32_t* hist, cudaStream_t st);
 int moegps_launch_plan(moegps_ctx* ctx, const int32_t* pred, int32_t* replicas, int32_t* slot_off,

@@ -354,21 +354,32 @@ rank_copy_kernel(const uint4* __restrict__ x, int T, int K, int chunks /* D*2/16
                  row_pair, xp, status);
 }
 
-// Dispatch after moegps_route_prepare: the count matrix (one column per router CTA, i.e. per
-// `rows_per` consecutive tokens, expert-major) and the slot row offsets exist already, so this single
-// kernel ranks, places and copies.  One warp per token: the stable rank of a pair = its expert's
-// counts over the earlier columns (a coalesced read by the warp) + the same-expert pairs of the
-// earlier tokens of its own column (the K experts of one token are distinct, so its own pairs never
-// count).  The first S blocks also mark the padding rows of one slot each with -1.
+// Dispatch after moegps_route_prepare: the count matrix exists already (one column per router CTA,
+// i.e. per `rows_per` consecutive tokens, expert-major), so this single kernel derives the offsets,
+// ranks, places and copies.  Every block first rebuilds the slot row offsets in its shared memory from
+// the finished histogram and the plan (a few hundred integer operations, cheaper than a launch or a
+// grid-wide hand-over; block 0 also stores them for the GEMMs).  Then one warp per token: the stable
+// rank of a pair = its expert's counts over the earlier columns (a coalesced read by the warp) + the
+// same-expert pairs of the earlier tokens of its own column (the K experts of one token are distinct,
+// so its own pairs never count).  The first S blocks also mark the padding rows of one slot each
+// with -1.
 __global__ void __launch_bounds__(kThreads)
 rank_copy_prepared_kernel(const uint4* __restrict__ x, int T, int K, int chunks, const int32_t* __restrict__ topk_idx,
-                          int E, int S, int64_t Rcap, const int32_t* __restrict__ seg_cnt, int nsub, int rows_per,
-                          const int32_t* __restrict__ hist, const int32_t* __restrict__ replicas,
-                          const int32_t* __restrict__ slot_off, const int32_t* __restrict__ slot_row_off,
+                          int E, int S, int A, int64_t Rcap, const int32_t* __restrict__ seg_cnt, int nsub,
+                          int rows_per, const int32_t* __restrict__ hist, const int32_t* __restrict__ replicas,
+                          const int32_t* __restrict__ slot_off, int32_t* __restrict__ slot_row_off,
                           int32_t* __restrict__ pair_row, int32_t* __restrict__ row_pair, uint4* __restrict__ xp,
                           int32_t* __restrict__ status) {
+  __shared__ int32_t s_row_off[kMaxS + 1];
+  __shared__ int32_t s_padded[kMaxS];
+  __shared__ int32_t s_warp_tot[kThreads / 32];
   __shared__ int pad_begin, pad_end;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  slot_offsets::build_slot_row_off<kThreads>(E, S, A, hist, replicas, slot_off, nullptr, s_padded, s_warp_tot,
+                                             s_row_off, status);
+  __syncthreads();
+  if (blockIdx.x == 0)
+    for (int s = threadIdx.x; s <= S; s += kThreads) slot_row_off[s] = s_row_off[s];
   // ---- padding rows of slots blockIdx.x, blockIdx.x + gridDim.x, ... ----
   for (int b = blockIdx.x; b < S; b += gridDim.x) {
     if (threadIdx.x == 0) { pad_begin = 0; pad_end = 0; }
@@ -380,8 +391,8 @@ rank_copy_prepared_kernel(const uint4* __restrict__ x, int T, int K, int chunks,
         const long long n = hist[e];
         const int rho = b - so;
         const int load = (int)(((long long)(rho + 1) * n) / r - ((long long)rho * n) / r);
-        pad_begin = slot_row_off[b] + load;
-        pad_end = slot_row_off[b + 1];
+        pad_begin = s_row_off[b] + load;
+        pad_end = s_row_off[b + 1];
       }
     }
     __syncthreads();
@@ -390,7 +401,7 @@ rank_copy_prepared_kernel(const uint4* __restrict__ x, int T, int K, int chunks,
     __syncthreads();
   }
   // ---- and the rows behind the last slot ----
-  for (int64_t row = (int64_t)slot_row_off[S] + (int64_t)blockIdx.x * kThreads + threadIdx.x; row < Rcap;
+  for (int64_t row = (int64_t)s_row_off[S] + (int64_t)blockIdx.x * kThreads + threadIdx.x; row < Rcap;
        row += (int64_t)gridDim.x * kThreads)
     if (row >= 0) row_pair[row] = -1;
   const int t = blockIdx.x * kWarpsPerBlock + warp;
@@ -418,7 +429,7 @@ rank_copy_prepared_kernel(const uint4* __restrict__ x, int T, int K, int chunks,
       }
     }
   }
-  place_and_copy(x, t, K, chunks, S, Rcap, my_e, my_rank, hist, replicas, slot_off, nullptr, slot_row_off, pair_row,
+  place_and_copy(x, t, K, chunks, S, Rcap, my_e, my_rank, hist, replicas, slot_off, nullptr, s_row_off, pair_row,
                  row_pair, xp, status);
 }
 
@@ -473,14 +484,14 @@ int moegps_launch_dispatch(moegps_ctx* ctx, const void* x, const int32_t* topk_i
 
 int moegps_launch_dispatch_prepared(moegps_ctx* ctx, const void* x, const int32_t* topk_idx, const int32_t* hist,
                                     const int32_t* replicas, const int32_t* slot_off,
-                                    const int32_t* slot_row_off, int32_t* row_pair, int32_t* pair_row, void* xp,
+                                    int32_t* slot_row_off, int32_t* row_pair, int32_t* pair_row, void* xp,
                                     const void* workspace, cudaStream_t st) {
   const moegps_shape_t& s = ctx->shape;
   const int rows_per = moegps_route_rows_per_cta(ctx);
   const int nsub = (s.T + 127) / 128 * (128 / rows_per);
   const int tblocks = (s.T + kWarpsPerBlock - 1) / kWarpsPerBlock;
   rank_copy_prepared_kernel<<<tblocks, kThreads, 0, st>>>(
-      static_cast<const uint4*>(x), s.T, s.K, s.D / 8, topk_idx, s.E, s.S, moegps_rcap_of(s),
+      static_cast<const uint4*>(x), s.T, s.K, s.D / 8, topk_idx, s.E, s.S, s.row_align, moegps_rcap_of(s),
       static_cast<const int32_t*>(workspace), nsub, rows_per, hist, replicas, slot_off, slot_row_off, pair_row, row_pair,
       static_cast<uint4*>(xp), ctx->d_status);
   MOEGPS_AFTER_LAUNCH(ctx);

@@ -21,17 +21,17 @@
 // Selection: L lanes per token select by shuffles (route_epilogue.cuh), L chosen so that the rows the
 // CTA owns occupy all sixteen warps in one pass.  When the caller asks for it, the per-expert token
 // counts (Eq. 1's n_e) are accumulated on the way: every selection bumps a shared-memory counter of
-// its CTA; each CTA adds its non-zero counters to accumulators that belong to the context (integer
-// atomics: deterministic) and draws a ticket; the CTA that draws the last one copies the sums to the
-// caller's histogram and leaves accumulators and ticket at zero for the next call - no memset, no
-// second kernel.  In the fused form (moegps_route_prepare) every CTA also stores its counters as one
-// column of the count matrix that dispatch ranks pairs with, and the last CTA derives the slot row
-// offsets from the finished histogram, so that dispatch is a single launch.
+// its CTA; each CTA adds its counters to 64-bit accumulators that belong to the context with one
+// atomic per expert (the count in the low half, an arrival mark in the high half; integer atomics:
+// deterministic); the thread whose atomic returns the last arrival for its expert holds the finished
+// count, stores it to the caller's histogram and zeroes the accumulator for the next call - no
+// memset, no fence, no second kernel.  In the fused form (moegps_route_prepare) every CTA also stores
+// its counters as one column of the count matrix that the dispatch step ranks pairs with, so that
+// dispatch is a single launch.
 // Warp roles in the main loop: warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
 // warps 2..5 = drain.  Every mbarrier wait is bounded.
 #include "common.cuh"
 #include "route_epilogue.cuh"
-#include "slot_offsets.cuh"
 #include "sm100.cuh"
 
 bool moegps_make_tmap_2d(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
@@ -165,10 +165,10 @@ __global__ void __launch_bounds__(kThreads, 1)
 route_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
              const RouteParams p, const float* __restrict__ bias, int32_t* __restrict__ topk_idx,
              float* __restrict__ topk_w, float* __restrict__ logits_out, int32_t* __restrict__ hist,
-             int32_t* __restrict__ acc /* context-owned: [256] sums + ticket at [256] */,
-             const moegps_route_fused fused, int S, int row_align, int32_t* __restrict__ status) {
+             unsigned long long* __restrict__ acc /* context-owned: [256] (arrivals, sum), zero between calls */,
+             int32_t* __restrict__ seg_cnt /* [E][CTAs] count matrix of the dispatch step, or nullptr */,
+             int32_t* __restrict__ status) {
   __shared__ int32_t cta_hist[256];       // this CTA's share of the histogram (used when hist != nullptr)
-  __shared__ int32_t s_last;
   __shared__ float s_bias[256];           // fetched while the stream runs
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -313,35 +313,18 @@ route_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     tc_fence_after_sync();
     tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
   }
-  if (hist) {
+  if (hist && (int)threadIdx.x < p.E) {
+    // One 64-bit atomic per expert and CTA adds this CTA's count (low half) and marks its arrival
+    // (high half); the thread whose atomic returns the last arrival holds the finished count.
     const int n_ctas = (int)(gridDim.x * gridDim.y);
     const int sub = (int)blockIdx.x * p.ks + (int)rank;          // this CTA's column of the count matrix
-    for (int e = threadIdx.x; e < p.E; e += kThreads) {
-      const int c = cta_hist[e];
-      if (fused.seg_cnt) fused.seg_cnt[(int64_t)e * n_ctas + sub] = c;
-      if (c) atomicAdd(&acc[e], c);
-    }
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) s_last = atomicAdd(&acc[256], 1) == n_ctas - 1;
-    __syncthreads();
-    if (s_last) {                 // every CTA's sums are in: publish them and leave the accumulators at zero
-      __threadfence();
-      for (int e = threadIdx.x; e < p.E; e += kThreads) {
-        const int h = atomicExch(&acc[e], 0);
-        hist[e] = h;
-        cta_hist[e] = h;          // (re-used as the finished histogram for the offsets below)
-      }
-      if (threadIdx.x == 0) acc[256] = 0;
-      if (fused.seg_cnt) {
-        // slot row offsets of the dispatch step (they depend on the finished histogram only);
-        // the ring memory is free by now and serves as scratch
-        int32_t* padded = reinterpret_cast<int32_t*>(smem);
-        int32_t* warp_tot = padded + slot_offsets::kMaxS;
-        __syncthreads();
-        slot_offsets::build_slot_row_off<kThreads>(p.E, S, row_align, cta_hist, fused.replicas, fused.slot_off,
-                                                   nullptr, padded, warp_tot, fused.slot_row_off, status);
-      }
+    const int e = (int)threadIdx.x;
+    const int c = cta_hist[e];
+    if (seg_cnt) seg_cnt[(int64_t)e * n_ctas + sub] = c;
+    const unsigned long long old = atomicAdd(&acc[e], (1ull << 32) | (unsigned long long)(uint32_t)c);
+    if ((int)(old >> 32) == n_ctas - 1) {
+      hist[e] = (int)(uint32_t)old + c;
+      acc[e] = 0;                       // zero again for the next call
     }
   }
 }
@@ -364,7 +347,7 @@ int route_split(const moegps_ctx* ctx) {
 int moegps_route_rows_per_cta(const moegps_ctx* ctx) { return BM / route_split(ctx); }
 
 int moegps_launch_route(moegps_ctx* ctx, const void* x, const void* wr, const float* bias, int32_t* topk_idx,
-                        float* topk_w, float* logits_out, int32_t* hist, const moegps_route_fused* fused,
+                        float* topk_w, float* logits_out, int32_t* hist, int32_t* seg_cnt,
                         cudaStream_t st) {
   const moegps_shape_t& s = ctx->shape;
   RouteParams p;
@@ -418,10 +401,8 @@ int moegps_launch_route(moegps_ctx* ctx, const void* x, const void* wr, const fl
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  const moegps_route_fused none = {nullptr, nullptr, nullptr, nullptr};
   cudaError_t e = cudaLaunchKernelEx(&cfg, route_kernel, ctx->tm_rx, ctx->tm_rw, p, bias, topk_idx, topk_w,
-                                     logits_out, hist, ctx->d_route_acc, fused ? *fused : none, (int)s.S,
-                                     (int)s.row_align, ctx->d_status);
+                                     logits_out, hist, ctx->d_route_acc, seg_cnt, ctx->d_status);
   ctx->launches += 1;
   if (e != cudaSuccess) {
     ctx->last_cuda_error = (int)e;

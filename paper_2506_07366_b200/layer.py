@@ -52,15 +52,14 @@ class MoeLayer:
         self._planned = True
 
     def forward(self, x, stream=None, out=None):
-        """route (+ histogram + the counts and offsets dispatch needs: one kernel) -> dispatch (one
-        kernel) -> expert_ffn -> combine on device tensor x [T, D]: five launches.
+        """route (+ histogram + the counts dispatch ranks with: one kernel) -> dispatch (offsets, ranks,
+        copies: one kernel) -> expert_ffn -> combine on device tensor x [T, D]: five launches.
         The result goes to `out` (bf16 [T, D]) if given, else to the layer's own buffer."""
         if not self._planned:
             raise RuntimeError("call plan(predicted_hist) before forward()")
         c = self.ctx
         out = self.out if out is None else out
-        c.route_prepare(x, self.w_router, self.bias, self.replicas, self.slot_off, self.topk_idx, self.topk_w,
-                        self.hist, self.slot_row_off, self.workspace, stream)
+        c.route_prepare(x, self.w_router, self.bias, self.topk_idx, self.topk_w, self.hist, self.workspace, stream)
         c.dispatch_prepared(x, self.topk_idx, self.hist, self.replicas, self.slot_off, self.slot_row_off,
                             self.row_pair, self.pair_row, self.xp, self.workspace, stream)
         c.expert_ffn(self.xp, self.slot_row_off, self.slot_expert, self.w_gate, self.w_up,

@@ -236,7 +236,7 @@ FUSED_CASES = [
 
 @pytest.mark.parametrize("w,A", FUSED_CASES, ids=lambda v: v if isinstance(v, int) else f"{v.name}-T{v.T}-D{v.D}-E{v.E}-K{v.K}")
 def test_route_prepare_and_dispatch_prepared_equal_the_separate_calls_and_the_oracle(w, A):
-    """The two-launch form (router also produces the counts and offsets dispatch needs) against the
+    """The two-launch form (router also produces the counts dispatch ranks with) against the
     four-launch form, bit for bit, and against the oracle; twice in a row with different batches,
     because the router's accumulators live in the context and must be back at zero after every call."""
     wr, bias = wl.router(w, "cpu")
@@ -263,7 +263,7 @@ def test_route_prepare_and_dispatch_prepared_equal_the_separate_calls_and_the_or
         idx_b, wt_b, hist_b = poison_i32(w.T, w.K), torch.full((w.T, w.K), float("nan"), device=DEV), poison_i32(w.E)
         sro_b, rp_b, pr_b = poison_i32(w.S + 1), poison_i32(shape.Rcap), poison_i32(w.T, w.K)
         xp_b = torch.full((shape.Rcap, w.D), 0x5A5A, dtype=torch.int16, device=DEV).view(torch.bfloat16)
-        ctx.route_prepare(xd, wrd, bd, rep, so, idx_b, wt_b, hist_b, sro_b, ws_b)
+        ctx.route_prepare(xd, wrd, bd, idx_b, wt_b, hist_b, ws_b)
         ctx.dispatch_prepared(xd, idx_b, hist_b, rep, so, sro_b, rp_b, pr_b, xp_b, ws_b)
         ctx.check_status()
         for a, b, what in ((idx_a, idx_b, "topk_idx"), (wt_a, wt_b, "topk_w"), (hist_a, hist_b, "hist"),
@@ -276,14 +276,18 @@ def test_route_prepare_and_dispatch_prepared_equal_the_separate_calls_and_the_or
         assert np.array_equal(rp_b.cpu().numpy(), rp_ref) and np.array_equal(pr_b.cpu().numpy(), pr_ref)
 
 
-def test_route_prepare_without_tokens():
+def test_route_prepare_and_dispatch_prepared_without_tokens():
     shape = binding.Shape(0, 64, 64, 4, 2, 6, 0, 8)
     ctx = binding.Context(shape)
     hist, sro = poison_i32(4), poison_i32(7)
     ws = torch.zeros(binding.workspace_bytes(shape), dtype=torch.uint8, device=DEV)
-    ctx.route_prepare(torch.zeros(0, 64, dtype=torch.bfloat16, device=DEV), torch.zeros(4, 64, dtype=torch.bfloat16, device=DEV),
-                      None, i32([2, 2, 1, 1]), i32([0, 2, 4, 5, 6]), torch.zeros(0, 2, dtype=torch.int32, device=DEV),
-                      torch.zeros(0, 2, dtype=torch.float32, device=DEV), hist, sro, ws)
+    x = torch.zeros(0, 64, dtype=torch.bfloat16, device=DEV)
+    idx = torch.zeros(0, 2, dtype=torch.int32, device=DEV)
+    ctx.route_prepare(x, torch.zeros(4, 64, dtype=torch.bfloat16, device=DEV), None, idx,
+                      torch.zeros(0, 2, dtype=torch.float32, device=DEV), hist, ws)
+    ctx.dispatch_prepared(x, idx, hist, i32([2, 2, 1, 1]), i32([0, 2, 4, 5, 6]), sro,
+                          torch.zeros(shape.Rcap, dtype=torch.int32, device=DEV), idx.clone(),
+                          torch.zeros(shape.Rcap, 64, dtype=torch.bfloat16, device=DEV), ws)
     ctx.check_status()
     assert hist.tolist() == [0] * 4 and sro.tolist() == [0] * 7
 
