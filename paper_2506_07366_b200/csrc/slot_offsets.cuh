@@ -1,4 +1,4 @@
-// Slot row offsets of the dispatch step (shared by the dispatch kernels and the router's fused tail):
+// Slot row offsets of the dispatch step (shared by the three dispatch kernels that derive them):
 // how an expert's pairs are split over its copies, the rows each slot reserves, and their prefix sum.
 #pragma once
 
