@@ -139,6 +139,11 @@ PLAN_CASES = [
     ([4, 2], 3, 0), ([2, 2], 3, 0), ([4, 2], 4, 0), ([0, 0, 0], 8, 0), ([5, 0, 1], 5, 0), ([3, 3, 3], 3, 0),
     ([100, 1, 1], 8, 3), ([100, 1], 8, 2), ([9000, 1000, 1000, 1000], 12, 0),
     ([2 ** 31 - 1, 2 ** 31 - 2, 5], 64, 0),
+    # ratios that differ by the least amount two fractions with denominators <= 1024 can differ by,
+    # 1 / (r1 r2), at the largest replica counts and counts the kernel supports, and exact ties there
+    ([2 ** 31 - 1, 2 ** 31 - 2], 1024, 0), ([1023 * 1024 + 1, 1023 * 1024, 1], 1024, 0),
+    ([511 * 512, 511 * 512 + 1, 511 * 512 - 1, 0], 1024, 0), ([2 ** 31 - 1, 2 ** 31 - 1, 2 ** 31 - 1], 1024, 0),
+    ([2 ** 31 - 1] + [2 ** 30] * 3 + [1] * 60, 1024, 700), ([6, 4, 3, 2, 12], 1000, 0),
 ]
 
 
