@@ -325,9 +325,13 @@ class Bench:
         that buffer, so the call's inputs come from HBM and its stores evict nothing dirty.  The
         interval between the two events also holds the launch latency of the stream and the event
         records themselves (`event_pair` = the same measurement with nothing in between; calls that
-        launch two kernels pay the gap twice).  These numbers explain the step time; they are not
-        part of the timed step."""
+        launch two kernels pay the gap twice).  The loop starts after a one-second pause: right after
+        a run of steps the chip is still at its power cap (SM clock near 1.4 GHz instead of 1.97) and
+        these short latency-bound calls would read up to 1.5x longer.  These numbers explain the step
+        time; they are not part of the timed step."""
         w, L, c = self.w, self.layer, self.ctx
+        torch.cuda.synchronize()
+        time.sleep(1.0)
         stream = torch.cuda.current_stream()
         evict = torch.zeros(128 << 20, dtype=torch.float32, device=self.dev)
         R, T, D, F, E, K = w.R, w.T, w.D, w.F, w.E, w.K
