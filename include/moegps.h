@@ -33,6 +33,9 @@
  *    out-of-range read or write is made for it) and MOEGPS_ERR_BAD_INDEX is recorded.
  *  - Weight layouts are "output features x input features", so both GEMM operands are contiguous
  *    along the contraction.
+ *  - If the environment variable MOEGPS_TRACE is set (and not "0") when a context is created, every
+ *    kernel launch made through that context is logged to stderr (ordinal, launcher, shape).  Host
+ *    side only; nothing on the device changes.
  */
 #ifndef MOEGPS_H_
 #define MOEGPS_H_

@@ -2,6 +2,8 @@
 // Every step validates its arguments here and launches nothing when they are wrong.
 #include <new>
 
+#include <stdlib.h>
+
 #include "common.cuh"
 
 namespace {
@@ -51,6 +53,8 @@ int moegps_create(moegps_ctx_t** out, const moegps_shape_t* shape, int device) {
   ctx->route_attr_done = false;
   ctx->dispatch_attr_done = false;
   ctx->pack_attr_done = false;
+  const char* trace = getenv("MOEGPS_TRACE");
+  ctx->trace = trace && trace[0] && trace[0] != '0';
   ctx->d_status = nullptr;
   ctx->d_route_acc = nullptr;
   int prev = 0;

@@ -5,6 +5,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdio.h>
 
 #include "moegps.h"
 
@@ -32,7 +33,16 @@ struct moegps_ctx {
   bool route_attr_done;
   bool dispatch_attr_done;
   bool pack_attr_done;
+  bool trace;               // MOEGPS_TRACE was set when the context was created: log every launch to stderr
 };
+
+// Host-side launch log (off unless the environment asked for it): ordinal, launcher, shape.
+inline void moegps_trace_launch(const moegps_ctx* ctx, const char* where) {
+  if (!ctx->trace) return;
+  const moegps_shape_t& s = ctx->shape;
+  fprintf(stderr, "[moegps] launch %lld %s T=%d D=%d F=%d E=%d K=%d S=%d A=%d\n", (long long)ctx->launches, where, s.T, s.D,
+          s.F, s.E, s.K, s.S, s.row_align);
+}
 
 #define MOEGPS_CUDA_TRY(ctx, expr)                                   \
   do {                                                               \
@@ -47,6 +57,7 @@ struct moegps_ctx {
 #define MOEGPS_AFTER_LAUNCH(ctx)                                     \
   do {                                                               \
     (ctx)->launches += 1;                                            \
+    moegps_trace_launch((ctx), __func__);                            \
     cudaError_t _e = cudaGetLastError();                             \
     if (_e != cudaSuccess) {                                         \
       (ctx)->last_cuda_error = (int)_e;                              \

@@ -404,6 +404,7 @@ int moegps_launch_route(moegps_ctx* ctx, const void* x, const void* wr, const fl
   cudaError_t e = cudaLaunchKernelEx(&cfg, route_kernel, ctx->tm_rx, ctx->tm_rw, p, bias, topk_idx, topk_w,
                                      logits_out, hist, ctx->d_route_acc, seg_cnt, ctx->d_status);
   ctx->launches += 1;
+  moegps_trace_launch(ctx, __func__);
   if (e != cudaSuccess) {
     ctx->last_cuda_error = (int)e;
     return MOEGPS_ERR_CUDA;

@@ -181,6 +181,23 @@ def run_plan(pred, S, c_max):
     assert int(bound.item()) == b_ref
 
 
+def test_trace_logs_every_launch_to_stderr(capfd, monkeypatch):
+    """MOEGPS_TRACE: a host-side log line per kernel launch, read when the context is created."""
+    monkeypatch.setenv("MOEGPS_TRACE", "1")
+    ctx = binding.Context(binding.Shape(8, 64, 64, 4, 1, 6, 0, 1))
+    monkeypatch.delenv("MOEGPS_TRACE")
+    quiet = binding.Context(binding.Shape(8, 64, 64, 4, 1, 6, 0, 1))
+    capfd.readouterr()
+    args = lambda: (i32([5, 1, 1, 1]), 6, poison_i32(4), poison_i32(5), poison_i32(6), poison_i32(1))  # noqa: E731
+    quiet.plan(*args())
+    assert "[moegps]" not in capfd.readouterr().err
+    n0 = ctx.launch_count()
+    ctx.plan(*args())
+    ctx.check_status()
+    err = capfd.readouterr().err
+    assert f"[moegps] launch {n0 + 1} moegps_launch_plan T=8 D=64 F=64 E=4 K=1 S=6 A=1" in err
+
+
 def test_plan_rejects_wrong_slot_count():
     ctx = binding.Context(binding.Shape(8, 64, 64, 4, 1, 6, 0, 1))
     n0 = ctx.launch_count()
